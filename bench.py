@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the GAF filter-accumulate hot path (Algorithm 1 + Eq. 5).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one whole gaf_filter_accumulate call over one batch of K synthetic
+micro-gradients (seed, K-1 cosine-distance tests, accepts, final division).
+The default workload is configuration 2 (ResNet18-sized gradients, D=11,227,812
+fp32, K=4, tau=0.97).  The path does not shard, so N > 1 runs N independent
+replicas, one per GPU (no collective on the data path); time is the max over
+ranks and the value is the aggregate over all replicas.
+
+Rank 0 prints ONE JSON line.  `value` is micro-gradient GB/s: bytes of input
+gradients consumed per second (K * elem_bytes * D per step), inputs resident in
+HBM.  `roofline` reports the HBM bytes the schedule must move (by its byte model,
+for the accept mask actually obtained) per second against the measured copy
+bandwidth of the box.  `e2e` is the same metric through the host-buffer entry
+point, pinned host memory in, results back to the host, copies inside the timed
+region.  `cpu_baseline` is the fp64 CPU oracle timed on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "gaf_filter_accumulate micro-gradient GB/s"
+UNIT = "GB/s"
+N_SETS = 4                       # rotating input sets: each step's inputs are cold in L2
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 4, 5],
+                    help="named configuration (2 is the one the metric is quoted on)")
+    ap.add_argument("--tau", type=float, default=0.97)
+    ap.add_argument("--schedule", type=int, default=0, help="0 auto, 1 stepwise, 2 persistent")
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def schedule_bytes(mask_in_order, K, D, b):
+    """HBM bytes the fused streaming schedule moves for a given accept pattern:
+    pass 0 reads the seed and candidate 1 and writes the running sum; pass t reads
+    the running sum and candidate t+1, plus gradient t and a write-back when t was
+    accepted; the last pass reads the running sum (plus the last gradient if
+    accepted) and writes g/c."""
+    if K == 1:
+        return (b + 4) * D
+    a = [int(x) for x in mask_in_order]          # a[t] for t = 1..K-1 at index t
+    total = 2 * b + 4
+    for t in range(1, K - 1):
+        total += 4 + b + a[t] * (b + 4)
+    total += 8 + a[K - 1] * b
+    return total * D
+
+
+# ---------------------------------------------------------------- clocks -----
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the
+    timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def sample(self):
+        nv = self.nv
+        self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+        for name, bit in (("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
+                          ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                          ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
+                          ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap),
+                          ("hw_power_brake", nv.nvmlClocksEventReasonHwPowerBrakeSlowdown)):
+            if bits & bit:
+                self.reasons.add(name)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.sample()
+            except Exception:
+                break
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        if self.ok and not self.samples:
+            try:
+                self.sample()
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------- CPU oracle leg ---
+
+def time_oracle(cfg: int, tau: float, seconds: float):
+    """The fp64 CPU oracle, as it stands, on the same workload (single thread)."""
+    import numpy as np  # noqa: F401
+    from oracle import gaf_oracle as orc
+    from paper_2412_18052_b200 import workloads
+
+    full = {1: 1_000_000, 2: workloads.RESNET18_100_NUMEL, 4: workloads.GPT2_SMALL_NUMEL,
+            5: 1_000_000_000}[cfg]
+    # configurations 4 and 5 are sampled at reduced D (same recipe) to bound the run
+    D = full if cfg in (1, 2) else min(full, 32_000_000)
+    w = workloads.config(cfg, device="cpu", D=None if D == full else D)
+    grads = [workloads.as_numpy_bits(g) for g in w.grads]
+    orc.filter_accumulate(grads, tau)                                  # warm (page in, compile)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        orc.filter_accumulate(grads, tau)
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds or reps >= 10_000:
+            break
+    per_call = dt / reps
+    gbs = w.K * w.elem_bytes * w.D / per_call / 1e9
+    sample = (f"configuration {cfg} recipe, K={w.K}, D={w.D:,} {w.dtype}"
+              f"{'' if D == full else ' (reduced from D=%d)' % full}, whole call repeated {reps}x "
+              f"({dt:.1f} s of CPU work)")
+    return gbs, per_call, sample
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, args.steps)
+    # each "step" of this arm is one oracle call on the bounded sample
+    budget = min(120.0, max(5.0, args.cpu_seconds))
+    gbs, per_call, sample = time_oracle(args.workload, args.tau, budget)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": per_call * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"configuration {args.workload}", "tau": args.tau},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ ours -----
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2412_18052_b200 as gaf
+    from paper_2412_18052_b200 import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = args.workload
+    n_sets = N_SETS if cfg in (1, 2) else (2 if cfg == 4 else 1)
+    sets = [workloads.config(cfg, device=dev, seed=(cfg - 1) + 1000 * i + 17 * rank) for i in range(n_sets)]
+    w0 = sets[0]
+    K, D, b = w0.K, w0.D, w0.elem_bytes
+    dtype_code = gaf.GAF_F32 if w0.dtype == "f32" else gaf.GAF_BF16
+    ws = gaf.new_workspace(K, D, dtype_code, device=dev)
+    macro = torch.empty(D, dtype=torch.float32, device=dev)
+    mask = torch.empty(K, dtype=torch.uint8, device=dev)
+    dist_out = torch.empty(K, dtype=torch.float32, device=dev)
+    count = torch.empty(1, dtype=torch.int32, device=dev)
+
+    def step(i):
+        gaf.gaf_filter_accumulate(sets[i % n_sets].grads, args.tau, ws, macro_out=macro, mask_out=mask,
+                                  dist_out=dist_out, count_out=count, schedule=args.schedule)
+
+    # accept pattern and byte model per input set (also a warm-up)
+    masks, bytes_per_set, launches_per_step = [], [], 0
+    for i in range(n_sets):
+        step(i)
+        launches_per_step = gaf.gaf_last_launch_count()
+        torch.cuda.synchronize()
+        m = mask.cpu().tolist()
+        masks.append(m)
+        bytes_per_set.append(schedule_bytes(m, K, D, b))
+        status = gaf.gaf_read_status(ws)
+        if status & gaf.GAF_STATUS_TIMEOUT:
+            raise SystemExit("device-side wait timed out during warm-up")
+    for i in range(max(3, args.warmup)):
+        step(i)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    steps = args.steps
+    sampler = ClockSampler(local)
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(steps):
+        step(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / steps
+    grad_bytes = K * b * D
+    value = world * grad_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # dominant kernel, timed per launch with events on the launching stream
+    n_launch_timed = min(steps, 200)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(n_launch_timed)]
+    for i, (a, z) in enumerate(evs):
+        a.record(); step(i); z.record()
+    torch.cuda.synchronize()
+    launch_ms = [a.elapsed_time(z) for a, z in evs]
+    avg_launch_ms = sum(launch_ms) / len(launch_ms)
+    avg_bytes = sum(bytes_per_set[i % n_sets] for i in range(n_launch_timed)) / n_launch_timed
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_kind = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_kind = 6650.0, "fallback"
+    achieved = avg_bytes / (avg_launch_ms * 1e-3) / 1e9
+    sustained = (sum(bytes_per_set[i % n_sets] for i in range(steps)) / steps) / (ms_per_step * 1e-3) / 1e9
+
+    # end to end through the host-buffer entry point
+    e2e = None
+    if args.e2e_steps > 0:
+        n_e2e = args.e2e_steps
+        host_sets = [[g.cpu().pin_memory() for g in s.grads] for s in sets[:2]]
+        staging = torch.empty(gaf.gaf_host_staging_bytes(K, D, dtype_code), dtype=torch.uint8, device=dev)
+        macro_h = torch.empty(D, dtype=torch.float32).pin_memory()
+        mask_h = torch.empty(K, dtype=torch.uint8).pin_memory()
+        dist_h = torch.empty(K, dtype=torch.float32).pin_memory()
+        count_h = torch.empty(1, dtype=torch.int32).pin_memory()
+
+        def e2e_step(i):
+            gaf.gaf_filter_accumulate_host(host_sets[i % len(host_sets)], args.tau, staging, ws, macro_h,
+                                           mask_h, dist_h, count_h, schedule=args.schedule)
+        for i in range(2):
+            e2e_step(i)
+        barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            e2e_step(i)                       # synchronises the stream itself
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * grad_bytes / (dt / n_e2e) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": grad_bytes, "d2h_bytes_per_step": 4 * D + K + 4 * K + 4,
+               "steps": n_e2e}
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            gbs, per_call, sample = time_oracle(cfg, args.tau, args.cpu_seconds)
+            cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": f"configuration {cfg}: K={K}, D={D}, {w0.dtype} inputs, tau={args.tau}, "
+                            f"shared+private Gaussian mixture" +
+                            (" with ResNet18 per-tensor scales" if cfg == 2 else ""),
+                "K": K, "D": D, "input_dtype": w0.dtype, "tau": args.tau,
+                "schedule": {0: "auto", 1: "stepwise", 2: "persistent"}[args.schedule],
+                "parallelism": "replicas only (the path does not shard)" if world > 1 else "1 GPU",
+                "l2": f"{n_sets} rotating input sets of {grad_bytes / 1e6:.0f} MB each (inputs of a step "
+                      f"exceed the 126 MB L2 and were last touched {n_sets - 1} steps earlier)"
+                      if n_sets > 1 else f"inputs of one step ({grad_bytes / 1e9:.1f} GB) exceed L2",
+                "accept_masks": masks,
+            },
+            "roofline": {
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_kind": f"of {peak_kind}",
+                "kernel": "persistent_kernel" if launches_per_step == 1 else "step_kernel x%d" % launches_per_step,
+                "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_launch_ms,
+                "sustained_achieved": sustained, "sustained_frac": sustained / peak,
+                "min_bytes_per_step": (K * b + 4) * D,
+            },
+            "e2e": e2e,
+            "gpu_launches": launches_per_step * steps,
+            "clocks": clocks,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

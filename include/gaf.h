@@ -1,0 +1,189 @@
+/*
+ * gaf.h -- C ABI of the Gradient Agreement Filtering hot path for NVIDIA B200
+ * (sm_100a).  Method: "Gradient Agreement Filtering", arxiv 2412.18052.
+ *
+ * Given K flattened micro-gradients of D parameters and a cosine-distance
+ * threshold tau, the library computes the cosine distance of Eq. 4 between the
+ * running sum of accepted micro-gradients and each incoming one, accepts or
+ * rejects it as Algorithm 1 states (D_c <= tau), and returns the filtered
+ * macro-gradient g/c of Eq. 5, the accept mask and the count c.  A K x K
+ * pairwise cosine-distance matrix (the quantity the paper's cosine-distance
+ * figures track) is provided for analysis.
+ *
+ * General conventions
+ *   - "device" pointers are CUDA global-memory addresses on the current device,
+ *     "host" pointers are ordinary process memory.
+ *   - The caller owns every buffer, including the workspace.  The library
+ *     allocates no device memory and keeps no state between calls other than
+ *     what lives in the caller's workspace.
+ *   - Every call is asynchronous on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and never synchronises, except
+ *     gaf_read_status and the *_host convenience call, which say so.
+ *   - Gradient buffers are read-only.  Every device pointer must be 16-byte
+ *     aligned (else GAF_ERR_ALIGN).  D need not be a multiple of anything.
+ *   - dtype: GAF_F32 = IEEE binary32, GAF_BF16 = bfloat16.  All arithmetic on
+ *     elements is binary32; sums are carried in binary64 from the thread level
+ *     up and reduced in a fixed order, so results are bitwise reproducible on
+ *     the same GPU model.  The scalar arithmetic of Eq. 4 and the comparison
+ *     with tau are binary64.
+ *   - Conventions where the paper is silent: a pair with a zero-norm member has
+ *     cos := 0 (distance 1); cos is clamped to [-1, 1]; a NaN distance is
+ *     rejected.  Either event sets a bit in the status word (see
+ *     gaf_read_status) and is otherwise not an error.
+ *   - Return value: GAF_OK or an error code; on an error detected on the host
+ *     nothing was launched.
+ */
+#ifndef GAF_H_
+#define GAF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GAF_MAX_K 64            /* largest number of micro-gradients per call */
+
+enum { GAF_F32 = 0, GAF_BF16 = 1 };
+
+enum {
+    GAF_OK = 0,
+    GAF_ERR_ARG = 1,            /* NULL pointer, K or D out of range, bad dtype/order/schedule */
+    GAF_ERR_ALIGN = 2,          /* a device pointer is not 16-byte aligned */
+    GAF_ERR_ALIAS = 3,          /* macro_out overlaps an input gradient */
+    GAF_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
+    GAF_ERR_CUDA = 5,           /* a CUDA runtime call failed (launch, copy) */
+    GAF_ERR_TIMEOUT = 6,        /* a bounded device-side wait ran out (see gaf_read_status) */
+    GAF_ERR_UNSUPPORTED = 7     /* the requested schedule cannot run on this device */
+};
+
+/* How gaf_filter_accumulate walks the K-1 sequential decisions of Algorithm 1.
+ * All schedules compute the same values in the same order of operations per
+ * element; they differ in launch structure only. */
+enum {
+    GAF_SCHED_AUTO = 0,         /* the library picks */
+    GAF_SCHED_STEPWISE = 1,     /* one launch per step; decisions stay on the device */
+    GAF_SCHED_PERSISTENT = 2    /* one cooperative launch; bulk-async shared-memory
+                                   pipeline that keeps prefetching across decisions */
+};
+
+/* Bits of the device status word. */
+enum {
+    GAF_STATUS_ZERO_NORM = 1,   /* some tested pair had a zero norm (distance set to 1) */
+    GAF_STATUS_NONFINITE = 2,   /* some sum was NaN or Inf */
+    GAF_STATUS_TIMEOUT = 4      /* a bounded wait expired; outputs are not valid */
+};
+
+/* Human-readable name of a return code.  Host only; never NULL. */
+const char *gaf_error_string(int code);
+
+/*
+ * Size in bytes of the workspace a call with these K, D, dtype needs (the
+ * maximum over the three operations).  Host only, touches no GPU.
+ * Errors: GAF_ERR_ARG for K outside [1, GAF_MAX_K], D < 0, bad dtype or NULL.
+ */
+int gaf_workspace_bytes(int K, int64_t D, int dtype, size_t *bytes_out);
+
+/*
+ * Prepare a workspace: clears its control block (asynchronous memset on the
+ * stream).  Needed once after allocation, and again after a call reported
+ * GAF_STATUS_TIMEOUT; calls that finish normally leave the workspace ready for
+ * the next call.  A workspace serves one call at a time: calls that share a
+ * workspace must be ordered on one stream.
+ *   workspace        device, 256-byte aligned, >= gaf_workspace_bytes(...)
+ */
+int gaf_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Cosine distance of Eq. 4 between two buffers:
+ *     D_c(x, y) = 1 - x.y / (|x| |y|).
+ *   x, y        device, D elements of `dtype` each
+ *   dist_out    device, 1 float
+ *   stats_out   device, 3 doubles {x.y, |x|^2, |y|^2}; may be NULL
+ */
+int gaf_cosdist(const void *x, const void *y, int64_t D, int dtype,
+                float *dist_out, double *stats_out,
+                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Algorithm 1 for one macrobatch followed by Eq. 5 (Section 3.1):
+ *     g <- g_{order[0]};  c <- 1
+ *     for t = 1 .. K-1, i = order[t]:
+ *         if D_c(g_i, g) <= tau:  g <- g + g_i;  c <- c + 1
+ *     macro_out <- g / c
+ * The test is against the running SUM g; the division happens once, at the end.
+ * The update/skip rule of the paper (skip the optimiser step when c == 1) is
+ * the caller's: read count_out.
+ *
+ *   grads       HOST array of K device pointers, D elements of `dtype` each
+ *   K           1 .. GAF_MAX_K (K == 1 returns the seed, c = 1)
+ *   D           >= 0
+ *   tau         threshold; tau >= 2 accepts everything (plain mean of Eq. 2),
+ *               tau < 0 rejects everything
+ *   order       HOST, permutation of 0..K-1, order[0] = seed s; NULL = identity
+ *               (the paper samples s at random: do that on the host)
+ *   macro_out   device, D floats (binary32 also for bf16 inputs); doubles as
+ *               the running sum during the call; must not overlap any input
+ *   mask_out    device, K bytes, by ORIGINAL index i: 1 accepted, 0 rejected;
+ *               mask[s] = 1
+ *   dist_out    device, K floats, by original index: D_c(g_i, g) at the moment
+ *               g_i was tested; dist[s] = 0; may be NULL
+ *   count_out   device, 1 int32: c
+ *   schedule    one of GAF_SCHED_*
+ */
+int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
+                          double tau, const int32_t *order,
+                          float *macro_out, uint8_t *mask_out, float *dist_out,
+                          int32_t *count_out,
+                          void *workspace, size_t workspace_bytes,
+                          int schedule, void *cuda_stream);
+
+/*
+ * The same operation for gradients that live in HOST memory (pinned memory
+ * makes the copies asynchronous and fast).  Copies each gradient to the device
+ * staging area, runs gaf_filter_accumulate, copies the results back and
+ * SYNCHRONISES the stream before returning.
+ *   grads_host      HOST array of K host pointers, D elements each
+ *   macro_out_host  host, D floats;  mask_out_host host, K bytes;
+ *   dist_out_host   host, K floats or NULL;  count_out_host host, 1 int32
+ *   staging         device, 256-byte aligned scratch for inputs and outputs,
+ *                   >= gaf_host_staging_bytes(K, D, dtype)
+ */
+int gaf_host_staging_bytes(int K, int64_t D, int dtype, size_t *bytes_out);
+int gaf_filter_accumulate_host(const void *const *grads_host, int K, int64_t D, int dtype,
+                               double tau, const int32_t *order,
+                               float *macro_out_host, uint8_t *mask_out_host,
+                               float *dist_out_host, int32_t *count_out_host,
+                               void *staging, size_t staging_bytes,
+                               void *workspace, size_t workspace_bytes,
+                               int schedule, void *cuda_stream);
+
+/*
+ * Pairwise cosine distances between K micro-gradients (Eq. 4 for every pair;
+ * what the paper's cosine-distance-over-training figures plot):
+ *     G = X X^T,  dist[i][j] = 1 - G_ij / (sqrt(G_ii) sqrt(G_jj)).
+ *   grads       HOST array of K device pointers
+ *   dist_out    device, K*K floats row-major; symmetric; diagonal 0 (1 for a
+ *               zero-norm gradient, whose whole row and column are 1)
+ *   gram_out    device, K*K doubles row-major (the Gram matrix); may be NULL
+ */
+int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype,
+                         float *dist_out, double *gram_out,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Read the device status word of the most recent call that used `workspace`.
+ * SYNCHRONISES the stream.  *status_out receives GAF_STATUS_* bits.  Returns
+ * GAF_ERR_TIMEOUT if the timeout bit is set, else GAF_OK.
+ */
+int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out);
+
+/* Number of kernel launches the most recent gaf_* call of this thread issued
+ * (host-side counter, for benchmarks). */
+int gaf_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GAF_H_ */

@@ -1,0 +1,212 @@
+"""Thin ctypes binding of the C ABI in ``include/gaf.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+PyTorch supplies device memory and the stream.  There is no fallback: if the
+shared library has not been built, or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+GAF_F32, GAF_BF16 = 0, 1
+GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_PERSISTENT = 0, 1, 2
+GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT = 1, 2, 4
+GAF_MAX_K = 64
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgaf.so")
+_lib = None
+
+EXPORTS = [
+    "gaf_error_string", "gaf_workspace_bytes", "gaf_workspace_init", "gaf_cosdist",
+    "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
+    "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count",
+]
+
+
+class GafError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib().gaf_error_string(code).decode()} (code {code})")
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2412_18052_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, dbl, sz = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
+                                 ctypes.c_size_t)
+        L.gaf_error_string.argtypes = [i32]
+        L.gaf_error_string.restype = ctypes.c_char_p
+        L.gaf_workspace_bytes.argtypes = [i32, i64, i32, ctypes.POINTER(sz)]
+        L.gaf_workspace_init.argtypes = [vp, sz, vp]
+        L.gaf_cosdist.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
+        L.gaf_filter_accumulate.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, i32, vp]
+        L.gaf_host_staging_bytes.argtypes = [i32, i64, i32, ctypes.POINTER(sz)]
+        L.gaf_filter_accumulate_host.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz,
+                                                 vp, sz, i32, vp]
+        L.gaf_pairwise_cosdist.argtypes = [vp, i32, i64, i32, vp, vp, vp, sz, vp]
+        L.gaf_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        L.gaf_last_launch_count.argtypes = []
+        for name in EXPORTS:
+            if name != "gaf_error_string":
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise GafError(code, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GAF_F32
+    if t.dtype == torch.bfloat16:
+        return GAF_BF16
+    raise TypeError(f"gradients must be float32 or bfloat16, got {t.dtype}")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr_array(tensors: Sequence[torch.Tensor]):
+    return (ctypes.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+def _order_array(order: Optional[Sequence[int]]):
+    if order is None:
+        return None
+    return (ctypes.c_int32 * len(order))(*[int(o) for o in order])
+
+
+def gaf_workspace_bytes(K: int, D: int, dtype: int) -> int:
+    out = ctypes.c_size_t()
+    _check(lib().gaf_workspace_bytes(K, D, dtype, ctypes.byref(out)), "gaf_workspace_bytes")
+    return out.value
+
+
+def gaf_host_staging_bytes(K: int, D: int, dtype: int) -> int:
+    out = ctypes.c_size_t()
+    _check(lib().gaf_host_staging_bytes(K, D, dtype, ctypes.byref(out)), "gaf_host_staging_bytes")
+    return out.value
+
+
+def new_workspace(K: int, D: int, dtype: int, device=None) -> torch.Tensor:
+    """Allocate (with torch) and initialise a workspace for calls up to this K."""
+    nbytes = gaf_workspace_bytes(K, D, dtype)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+    gaf_workspace_init(ws)
+    return ws
+
+
+def gaf_workspace_init(workspace: torch.Tensor) -> None:
+    _check(lib().gaf_workspace_init(workspace.data_ptr(), workspace.numel(), _stream()),
+           "gaf_workspace_init")
+
+
+def gaf_cosdist(x: torch.Tensor, y: torch.Tensor, workspace: torch.Tensor,
+                dist_out: Optional[torch.Tensor] = None,
+                stats_out: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Eq. 4 between two device tensors.  Returns (dist[1] float32, stats[3] float64)."""
+    assert x.numel() == y.numel() and x.dtype == y.dtype
+    if dist_out is None:
+        dist_out = torch.empty(1, dtype=torch.float32, device=x.device)
+    if stats_out is None:
+        stats_out = torch.empty(3, dtype=torch.float64, device=x.device)
+    _check(lib().gaf_cosdist(x.data_ptr(), y.data_ptr(), x.numel(), _dtype_code(x),
+                             dist_out.data_ptr(), stats_out.data_ptr(),
+                             workspace.data_ptr(), workspace.numel(), _stream()), "gaf_cosdist")
+    return dist_out, stats_out
+
+
+def gaf_filter_accumulate(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,
+                          order: Optional[Sequence[int]] = None,
+                          macro_out: Optional[torch.Tensor] = None,
+                          mask_out: Optional[torch.Tensor] = None,
+                          dist_out: Optional[torch.Tensor] = None,
+                          count_out: Optional[torch.Tensor] = None,
+                          schedule: int = GAF_SCHED_AUTO):
+    """Algorithm 1 + Eq. 5 on device tensors.  Returns (macro, mask, dist, count) device tensors."""
+    K, D = len(grads), grads[0].numel()
+    dev = grads[0].device
+    code = _dtype_code(grads[0])
+    for g in grads:
+        assert g.numel() == D and g.dtype == grads[0].dtype and g.is_contiguous()
+    if macro_out is None:
+        macro_out = torch.empty(D, dtype=torch.float32, device=dev)
+    if mask_out is None:
+        mask_out = torch.empty(K, dtype=torch.uint8, device=dev)
+    if dist_out is None:
+        dist_out = torch.empty(K, dtype=torch.float32, device=dev)
+    if count_out is None:
+        count_out = torch.empty(1, dtype=torch.int32, device=dev)
+    ptrs = _ptr_array(grads)
+    ordp = _order_array(order)
+    _check(lib().gaf_filter_accumulate(ctypes.cast(ptrs, ctypes.c_void_p), K, D, code, float(tau),
+                                       ordp and ctypes.cast(ordp, ctypes.c_void_p),
+                                       macro_out.data_ptr(), mask_out.data_ptr(), dist_out.data_ptr(),
+                                       count_out.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                       int(schedule), _stream()), "gaf_filter_accumulate")
+    return macro_out, mask_out, dist_out, count_out
+
+
+def gaf_filter_accumulate_host(grads_host: Sequence[torch.Tensor], tau: float,
+                               staging: torch.Tensor, workspace: torch.Tensor,
+                               macro_out_host: torch.Tensor, mask_out_host: torch.Tensor,
+                               dist_out_host: torch.Tensor, count_out_host: torch.Tensor,
+                               order: Optional[Sequence[int]] = None,
+                               schedule: int = GAF_SCHED_AUTO) -> None:
+    """Same operation on HOST tensors (pinned for speed); synchronises the stream."""
+    K, D = len(grads_host), grads_host[0].numel()
+    code = _dtype_code(grads_host[0])
+    ptrs = _ptr_array(grads_host)
+    ordp = _order_array(order)
+    _check(lib().gaf_filter_accumulate_host(
+        ctypes.cast(ptrs, ctypes.c_void_p), K, D, code, float(tau),
+        ordp and ctypes.cast(ordp, ctypes.c_void_p),
+        macro_out_host.data_ptr(), mask_out_host.data_ptr(), dist_out_host.data_ptr(),
+        count_out_host.data_ptr(), staging.data_ptr(), staging.numel(),
+        workspace.data_ptr(), workspace.numel(), int(schedule), _stream()),
+        "gaf_filter_accumulate_host")
+
+
+def gaf_pairwise_cosdist(grads: Sequence[torch.Tensor], workspace: torch.Tensor,
+                         dist_out: Optional[torch.Tensor] = None,
+                         gram_out: Optional[torch.Tensor] = None):
+    """K x K cosine-distance matrix (float32) and Gram matrix (float64) on the device."""
+    K, D = len(grads), grads[0].numel()
+    dev = grads[0].device
+    if dist_out is None:
+        dist_out = torch.empty(K, K, dtype=torch.float32, device=dev)
+    if gram_out is None:
+        gram_out = torch.empty(K, K, dtype=torch.float64, device=dev)
+    ptrs = _ptr_array(grads)
+    _check(lib().gaf_pairwise_cosdist(ctypes.cast(ptrs, ctypes.c_void_p), K, D, _dtype_code(grads[0]),
+                                      dist_out.data_ptr(), gram_out.data_ptr(),
+                                      workspace.data_ptr(), workspace.numel(), _stream()),
+           "gaf_pairwise_cosdist")
+    return dist_out, gram_out
+
+
+def gaf_read_status(workspace: torch.Tensor) -> int:
+    """Status bits of the latest call on this workspace (synchronises the stream)."""
+    out = ctypes.c_int()
+    rc = lib().gaf_read_status(workspace.data_ptr(), _stream(), ctypes.byref(out))
+    if rc not in (0, 6):
+        raise GafError(rc, "gaf_read_status")
+    return out.value
+
+
+def gaf_last_launch_count() -> int:
+    return lib().gaf_last_launch_count()

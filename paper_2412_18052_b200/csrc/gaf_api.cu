@@ -1,0 +1,314 @@
+// Host side of the C ABI declared in include/gaf.h: argument checks, workspace
+// carve-up and kernel launches.  No device memory is allocated here.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstring>
+
+#include "../../include/gaf.h"
+#include "gaf_device.cuh"
+#include "gaf_pairwise.cuh"
+#include "gaf_persistent.cuh"
+#include "gaf_stepwise.cuh"
+
+namespace {
+
+using namespace gaf;
+
+thread_local int g_launches = 0;
+
+struct DeviceInfo {
+    int sms = 0;
+    int coop = 0;
+    int smem_optin = 0;
+};
+
+// Attributes of the current device (queried per call: two cheap driver lookups).
+bool device_info(DeviceInfo *out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&out->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&out->coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&out->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+        return false;
+    return out->sms > 0;
+}
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elem_bytes(int dtype) { return dtype == GAF_F32 ? 4 : 2; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t pairwise_extra_bytes(int K) {
+    const int tiles = (K + kGramTile - 1) / kGramTile;
+    const size_t pairs = size_t(tiles) * (tiles + 1) / 2;
+    return pairs * kGramMaxSlices * 64 * sizeof(double) + round_up(size_t(K) * K * sizeof(double), 256);
+}
+
+int check_workspace(const void *ws, size_t have, size_t need) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || have < need) return GAF_ERR_WORKSPACE;
+    return GAF_OK;
+}
+
+// CTAs for a streaming kernel of `threads` threads that handles 8 elements per
+// thread and iteration: two per SM, fewer when D is small.
+int stream_grid(int64_t D, int threads, int sms) {
+    int64_t need = (D / kOct + threads - 1) / threads;
+    int64_t cap = int64_t(sms) * 2;
+    if (cap > kMaxCtas) cap = kMaxCtas;
+    if (need < 1) need = 1;
+    return int(need < cap ? need : cap);
+}
+
+template <typename T>
+int launch_stepwise(const void *const *g, int K, int64_t D, double tau, const int32_t *ord,
+                    float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
+                    Control *ctl, double *partials, int sms, cudaStream_t st) {
+    const int grid = stream_grid(D, kStepThreads, sms);
+    StepArgs a{};
+    a.acc = macro_out; a.D = D; a.ctl = ctl; a.partials = partials; a.tau = tau;
+    a.mask_out = mask_out; a.dist_out = dist_out; a.count_out = count_out; a.K = K;
+    a.seed_index = ord[0];
+    a.g_seed = g[ord[0]];
+    if (K == 1) {
+        step_kernel<T, kOnly><<<grid, kStepThreads, 0, st>>>(a);
+        ++g_launches;
+        return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+    }
+    a.t = 0; a.g_next = g[ord[1]]; a.i_next = ord[1];
+    step_kernel<T, kFirst><<<grid, kStepThreads, 0, st>>>(a);
+    ++g_launches;
+    for (int t = 1; t <= K - 2; ++t) {
+        a.t = t; a.g_cur = g[ord[t]]; a.g_next = g[ord[t + 1]]; a.i_next = ord[t + 1];
+        step_kernel<T, kMid><<<grid, kStepThreads, 0, st>>>(a);
+        ++g_launches;
+    }
+    a.t = K - 1; a.g_cur = g[ord[K - 1]]; a.g_next = nullptr; a.i_next = -1;
+    step_kernel<T, kLast><<<grid, kStepThreads, 0, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int check_grads(const void *const *grads, int K, int64_t D, int dtype) {
+    if (!grads || K < 1 || K > GAF_MAX_K || D < 0) return GAF_ERR_ARG;
+    if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
+    for (int i = 0; i < K; ++i) {
+        if (!grads[i]) return GAF_ERR_ARG;
+        if (!aligned16(grads[i])) return GAF_ERR_ALIGN;
+    }
+    return GAF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *gaf_error_string(int code) {
+    switch (code) {
+        case GAF_OK: return "ok";
+        case GAF_ERR_ARG: return "invalid argument";
+        case GAF_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case GAF_ERR_ALIAS: return "macro_out overlaps an input gradient";
+        case GAF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case GAF_ERR_CUDA: return "CUDA runtime error";
+        case GAF_ERR_TIMEOUT: return "device-side wait timed out";
+        case GAF_ERR_UNSUPPORTED: return "schedule not supported on this device";
+        default: return "unknown error code";
+    }
+}
+
+int gaf_last_launch_count(void) { return g_launches; }
+
+int gaf_workspace_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {
+    if (!bytes_out || K < 1 || K > GAF_MAX_K || D < 0) return GAF_ERR_ARG;
+    if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
+    *bytes_out = round_up(kExtraOffset + pairwise_extra_bytes(K), 256);
+    return GAF_OK;
+}
+
+int gaf_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
+    g_launches = 0;
+    if (cudaMemsetAsync(workspace, 0, kControlBytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return GAF_ERR_CUDA;
+    return GAF_OK;
+}
+
+int gaf_cosdist(const void *x, const void *y, int64_t D, int dtype, float *dist_out,
+                double *stats_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    g_launches = 0;
+    if (!x || !y || !dist_out || D < 0) return GAF_ERR_ARG;
+    if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
+    if (!aligned16(x) || !aligned16(y)) return GAF_ERR_ALIGN;
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    CosArgs a{x, y, D, reinterpret_cast<Control *>(base),
+              reinterpret_cast<double *>(base + kPartialsOffset), dist_out, stats_out};
+    const int grid = stream_grid(D, kStepThreads, di.sms);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (dtype == GAF_F32) cosdist_kernel<float><<<grid, kStepThreads, 0, st>>>(a);
+    else cosdist_kernel<__nv_bfloat16><<<grid, kStepThreads, 0, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype, double tau,
+                          const int32_t *order, float *macro_out, uint8_t *mask_out,
+                          float *dist_out, int32_t *count_out, void *workspace,
+                          size_t workspace_bytes, int schedule, void *cuda_stream) {
+    g_launches = 0;
+    if (int rc = check_grads(grads, K, D, dtype)) return rc;
+    if (!macro_out || !mask_out || !count_out) return GAF_ERR_ARG;
+    if (schedule != GAF_SCHED_AUTO && schedule != GAF_SCHED_STEPWISE && schedule != GAF_SCHED_PERSISTENT)
+        return GAF_ERR_ARG;
+    if (tau != tau) return GAF_ERR_ARG;
+    if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
+    int32_t ord[GAF_MAX_K];
+    {
+        bool seen[GAF_MAX_K] = {false};
+        for (int t = 0; t < K; ++t) {
+            int32_t i = order ? order[t] : t;
+            if (i < 0 || i >= K || seen[i]) return GAF_ERR_ARG;
+            seen[i] = true;
+            ord[t] = i;
+        }
+    }
+    {
+        const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
+        for (int i = 0; i < K; ++i) {
+            const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
+            const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
+            if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
+        }
+    }
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    Control *ctl = reinterpret_cast<Control *>(base);
+    double *partials = reinterpret_cast<double *>(base + kPartialsOffset);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    if (schedule == GAF_SCHED_AUTO) {
+        schedule = (K >= 2 && persistent_supported(di.coop, di.smem_optin)) ? GAF_SCHED_PERSISTENT
+                                                                          : GAF_SCHED_STEPWISE;
+    }
+    if (schedule == GAF_SCHED_PERSISTENT) {
+        if (!persistent_supported(di.coop, di.smem_optin)) return GAF_ERR_UNSUPPORTED;
+        if (K >= 2) {
+            int rc = dtype == GAF_F32
+                ? launch_persistent<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
+                                           count_out, ctl, partials, di.sms, st)
+                : launch_persistent<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out,
+                                                   dist_out, count_out, ctl, partials, di.sms, st);
+            if (rc == GAF_OK) ++g_launches;
+            return rc;
+        }
+    }
+    return dtype == GAF_F32
+        ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
+                                 ctl, partials, di.sms, st)
+        : launch_stepwise<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
+                                         count_out, ctl, partials, di.sms, st);
+}
+
+int gaf_host_staging_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {
+    if (!bytes_out || K < 1 || K > GAF_MAX_K || D < 0) return GAF_ERR_ARG;
+    if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
+    const size_t g = round_up(size_t(D) * elem_bytes(dtype), 256);
+    *bytes_out = size_t(K) * g + round_up(size_t(D) * 4, 256) + 3 * 256;
+    return GAF_OK;
+}
+
+int gaf_filter_accumulate_host(const void *const *grads_host, int K, int64_t D, int dtype,
+                               double tau, const int32_t *order, float *macro_out_host,
+                               uint8_t *mask_out_host, float *dist_out_host,
+                               int32_t *count_out_host, void *staging, size_t staging_bytes,
+                               void *workspace, size_t workspace_bytes, int schedule,
+                               void *cuda_stream) {
+    g_launches = 0;
+    size_t need = 0;
+    if (int rc = gaf_host_staging_bytes(K, D, dtype, &need)) return rc;
+    if (!grads_host || !macro_out_host || !mask_out_host || !count_out_host) return GAF_ERR_ARG;
+    for (int i = 0; i < K; ++i) if (!grads_host[i]) return GAF_ERR_ARG;
+    if (int rc = check_workspace(staging, staging_bytes, need)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    auto *base = static_cast<unsigned char *>(staging);
+    const size_t gbytes = size_t(D) * elem_bytes(dtype), gstride = round_up(gbytes, 256);
+    const void *dev[GAF_MAX_K];
+    for (int i = 0; i < K; ++i) {
+        dev[i] = base + size_t(i) * gstride;
+        if (gbytes && cudaMemcpyAsync(base + size_t(i) * gstride, grads_host[i], gbytes,
+                                      cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return GAF_ERR_CUDA;
+    }
+    unsigned char *p = base + size_t(K) * gstride;
+    float *d_out = reinterpret_cast<float *>(p); p += round_up(size_t(D) * 4, 256);
+    uint8_t *d_mask = p; p += 256;
+    float *d_dist = reinterpret_cast<float *>(p); p += 256;
+    int32_t *d_count = reinterpret_cast<int32_t *>(p);
+    int rc = gaf_filter_accumulate(dev, K, D, dtype, tau, order, d_out, d_mask, d_dist, d_count,
+                                   workspace, workspace_bytes, schedule, cuda_stream);
+    if (rc != GAF_OK) return rc;
+    bool ok = true;
+    if (D) ok &= cudaMemcpyAsync(macro_out_host, d_out, size_t(D) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(mask_out_host, d_mask, K, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (dist_out_host)
+        ok &= cudaMemcpyAsync(dist_out_host, d_dist, size_t(K) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(count_out_host, d_count, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaStreamSynchronize(st) == cudaSuccess;
+    return ok ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype, float *dist_out,
+                         double *gram_out, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream) {
+    g_launches = 0;
+    if (int rc = check_grads(grads, K, D, dtype)) return rc;
+    if (!dist_out) return GAF_ERR_ARG;
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K)))
+        return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    GramArgs a{};
+    for (int i = 0; i < K; ++i) a.g[i] = grads[i];
+    a.K = K; a.D = D;
+    a.tiles = (K + kGramTile - 1) / kGramTile;
+    const int pairs = a.tiles * (a.tiles + 1) / 2;
+    a.partials = reinterpret_cast<double *>(base + kExtraOffset);
+    a.gram = reinterpret_cast<double *>(base + kExtraOffset +
+                                        size_t(pairs) * kGramMaxSlices * 64 * sizeof(double));
+    a.dist_out = dist_out; a.gram_out = gram_out;
+    a.ctl = reinterpret_cast<Control *>(base);
+    // D-slices: fill the machine about twice over all tile pairs, never more than there is work
+    int64_t slices = (int64_t(di.sms) * 2 + pairs - 1) / pairs;
+    const int64_t work = (D / 4 + kGramThreads - 1) / kGramThreads;
+    if (slices > work) slices = work;
+    if (slices > kGramMaxSlices) slices = kGramMaxSlices;
+    if (slices < 1) slices = 1;
+    a.slices = int(slices);
+    dim3 grid(a.slices, pairs);
+    if (dtype == GAF_F32) gram_tile_kernel<float><<<grid, kGramThreads, 0, st>>>(a);
+    else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
+    ++g_launches;
+    gram_finish_kernel<<<pairs, 256, 0, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out) {
+    if (!workspace || !status_out) return GAF_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const Control *ctl = static_cast<const Control *>(workspace);
+    int status = 0;
+    if (cudaMemcpyAsync(&status, &ctl->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return GAF_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return GAF_ERR_CUDA;
+    *status_out = status;
+    return (status & GAF_STATUS_TIMEOUT) ? GAF_ERR_TIMEOUT : GAF_OK;
+}
+
+}  // extern "C"

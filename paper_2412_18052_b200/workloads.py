@@ -128,11 +128,11 @@ def mixture(K: int, D: int, dtype: str, rho: Sequence[float], seed: int,
 
 
 def config(n: int, device: str = "cpu", D: Optional[int] = None,
-           K: Optional[int] = None) -> Workload:
+           K: Optional[int] = None, seed: Optional[int] = None) -> Workload:
     """Named configuration ``n`` (1..5).  ``D``/``K`` override the size for
     scaled-down copies of the same recipe (the tensor layout of configuration 2
-    is kept only at its native D)."""
-    seed = n - 1
+    is kept only at its native D); ``seed`` draws another instance of it."""
+    seed = n - 1 if seed is None else seed
     rgen = np.random.RandomState(seed)
     if n == 1:
         K_, D_, dtype, taus = 4, 1_000_000, "f32", [0.97]

@@ -1,0 +1,135 @@
+"""Parity harness: the CUDA library against the CPU oracle on the same bits.
+
+Tolerances (the bar the method's target states):
+  * cosine distances: 1e-5 absolute;
+  * accept masks: bit-exact, except that a decision whose oracle distance lies
+    within 1e-5 of tau may differ -- everything after such a flip legitimately
+    changes, so the oracle is re-run with that one decision forced to the GPU's
+    and the comparison continues against the replayed oracle;
+  * macro-gradient: relative L2 error 1e-6 for fp32 inputs, 1e-3 for bf16.
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+import paper_2412_18052_b200 as gaf
+from oracle import gaf_oracle as orc
+from paper_2412_18052_b200.workloads import as_numpy_bits
+
+DIST_ATOL = 1e-5
+MACRO_RTOL = {torch.float32: 1e-6, torch.bfloat16: 1e-3}
+
+
+def rel_l2(got: np.ndarray, want: np.ndarray) -> float:
+    """|got - want|_2 / |want|_2, accumulated in float64 chunk by chunk."""
+    num = den = 0.0
+    step = 1 << 24
+    for lo in range(0, want.size, step):
+        w = want[lo:lo + step].astype(np.float64)
+        g = got[lo:lo + step].astype(np.float64)
+        num += float(np.dot(g - w, g - w))
+        den += float(np.dot(w, w))
+    if den == 0.0:
+        return 0.0 if num == 0.0 else float("inf")
+    return (num / den) ** 0.5
+
+
+def oracle_with_replay(np_grads, tau, order, gpu_mask):
+    """Oracle result, re-run with forced decisions where the GPU legitimately
+    flipped a decision that sits within DIST_ATOL of tau.  Returns (result, replays)."""
+    K = len(np_grads)
+    steps = list(order) if order is not None else list(range(K))
+    forced = [-1] * K
+    replays = 0
+    while True:
+        r = orc.filter_accumulate(np_grads, tau, order=order, forced=forced if replays else None)
+        bad = None
+        for t in range(1, K):
+            i = steps[t]
+            if int(r.mask[i]) != int(gpu_mask[i]):
+                bad = (t, i)
+                break
+        if bad is None:
+            return r, replays
+        t, i = bad
+        assert abs(r.dist[i] - tau) < DIST_ATOL, (
+            f"mask differs at step {t} (gradient {i}) with oracle distance {r.dist[i]!r} "
+            f"not within {DIST_ATOL} of tau={tau}")
+        forced[t] = int(gpu_mask[i])
+        replays += 1
+        assert replays <= K
+
+
+def check_filter(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,
+                 order: Optional[Sequence[int]] = None, schedule: int = 0,
+                 np_grads=None, expect_status: Optional[int] = 0):
+    """Run gaf_filter_accumulate on the GPU and compare everything with the oracle.
+    Returns a dict of the measured errors."""
+    K, D = len(grads), grads[0].numel()
+    dev = grads[0].device
+    # guard bands around every output catch out-of-bounds writes
+    pad = 64
+    macro_buf = torch.full((D + 2 * pad,), 777.0, dtype=torch.float32, device=dev)
+    mask_buf = torch.full((K + 2 * pad,), 99, dtype=torch.uint8, device=dev)
+    dist_buf = torch.full((K + 2 * pad,), 777.0, dtype=torch.float32, device=dev)
+    count_buf = torch.full((1 + 2 * pad,), -5, dtype=torch.int32, device=dev)
+    macro, mask, dist, count = gaf.gaf_filter_accumulate(
+        grads, tau, workspace, order=order, schedule=schedule,
+        macro_out=macro_buf[pad:pad + D], mask_out=mask_buf[pad:pad + K],
+        dist_out=dist_buf[pad:pad + K], count_out=count_buf[pad:pad + 1])
+    status = gaf.gaf_read_status(workspace)
+    if expect_status is not None:
+        assert status == expect_status, f"device status {status}, expected {expect_status}"
+    for buf, fill, n in ((macro_buf, 777.0, D), (mask_buf, 99, K), (dist_buf, 777.0, K), (count_buf, -5, 1)):
+        assert bool((buf[:pad] == fill).all()) and bool((buf[pad + n:] == fill).all()), "guard band overwritten"
+
+    g_mask = mask.cpu().numpy()
+    g_dist = dist.cpu().numpy().astype(np.float64)
+    g_count = int(count.cpu().item())
+    g_macro = macro.cpu().numpy()
+
+    if np_grads is None:
+        np_grads = [as_numpy_bits(g) for g in grads]
+    r, replays = oracle_with_replay(np_grads, tau, order, g_mask)
+    assert g_mask.tolist() == r.mask.tolist()
+    assert g_count == r.count
+    finite = np.isfinite(r.dist)
+    dist_err = float(np.max(np.abs(g_dist[finite] - r.dist[finite]))) if finite.any() else 0.0
+    assert dist_err <= DIST_ATOL, f"distance error {dist_err}"
+    assert np.array_equal(np.isnan(g_dist), np.isnan(r.dist))
+    err = rel_l2(g_macro, r.out)
+    assert err <= MACRO_RTOL[grads[0].dtype], f"macro-gradient relative L2 error {err}"
+    return {"dist_err": dist_err, "macro_rel_l2": err, "replays": replays, "count": g_count,
+            "mask": g_mask.tolist(), "dist": g_dist.tolist()}
+
+
+def check_cosdist(x: torch.Tensor, y: torch.Tensor, workspace: torch.Tensor):
+    d, stats = gaf.gaf_cosdist(x, y, workspace)
+    want, (p, nx, ny) = orc.cosdist(as_numpy_bits(x), as_numpy_bits(y))
+    got = float(d.cpu().item())
+    assert abs(got - want) <= DIST_ATOL, (got, want)
+    st = stats.cpu().numpy()
+    scale = (nx * ny) ** 0.5
+    assert abs(st[0] - p) <= 1e-6 * scale + 1e-300
+    assert abs(st[1] - nx) <= 1e-6 * nx + 1e-300 and abs(st[2] - ny) <= 1e-6 * ny + 1e-300
+    return abs(got - want)
+
+
+def check_pairwise(grads: Sequence[torch.Tensor], workspace: torch.Tensor):
+    K = len(grads)
+    dist, gram = gaf.gaf_pairwise_cosdist(grads, workspace)
+    o_gram, o_dist = orc.pairwise_cosdist([as_numpy_bits(g) for g in grads])
+    g_dist = dist.cpu().numpy().astype(np.float64)
+    g_gram = gram.cpu().numpy()
+    err = float(np.max(np.abs(g_dist - o_dist)))
+    assert err <= DIST_ATOL, f"pairwise distance error {err}"
+    assert np.array_equal(g_dist, g_dist.T), "distance matrix not symmetric"
+    nrm = np.sqrt(np.abs(np.diag(o_gram)))
+    scale = np.outer(nrm, nrm) + 1e-300
+    assert float(np.max(np.abs(g_gram - o_gram) / scale)) <= 1e-5
+    for i in range(K):
+        assert g_dist[i, i] == (0.0 if o_gram[i, i] > 0 else 1.0)
+    return err

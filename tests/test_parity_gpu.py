@@ -1,0 +1,256 @@
+"""GPU parity tests proper: every entry point, through the C ABI, against the CPU
+oracle on the same seeded inputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2412_18052_b200 as gaf
+from paper_2412_18052_b200 import workloads
+from parity import check_cosdist, check_filter, check_pairwise
+
+pytestmark = pytest.mark.gpu
+
+SCHEDULES = [gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_PERSISTENT]
+SCHED_IDS = ["stepwise", "persistent"]
+DTYPES = ["f32", "bf16"]
+
+
+@pytest.fixture(scope="module")
+def ws():
+    return gaf.new_workspace(gaf.binding.GAF_MAX_K, 1 << 20, gaf.GAF_F32)
+
+
+def _mix(K, D, dtype, seed, rho=None, sigma=1e-3):
+    rng = np.random.RandomState(seed)
+    if rho is None:
+        rho = rng.uniform(-0.4, 0.9, size=K)
+    return workloads.mixture(K, D, dtype, list(rho), seed, device="cuda", sigma=sigma)
+
+
+# ------------------------------------------------------------------ Eq. 4 ----
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_cosdist_every_small_length(ws, dtype):
+    for D in list(range(0, 41)) + [63, 64, 65, 511, 4095, 4097]:
+        w = _mix(2, D, dtype, seed=100 + D, rho=[0.6, 0.3])
+        check_cosdist(w.grads[0], w.grads[1], ws)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("D", [1_000_003, 8 * 512 * 296 * 3 + 5])
+def test_cosdist_several_waves_and_ragged_tail(ws, dtype, D):
+    w = _mix(2, D, dtype, seed=7, rho=[0.2, -0.5])
+    err = check_cosdist(w.grads[0], w.grads[1], ws)
+    assert err < 1e-6
+
+
+def test_cosdist_stated_values(ws):
+    x = torch.randn(10_001, device="cuda")
+    for y, want in ((x.clone(), 0.0), (-x, 2.0)):
+        d, _ = gaf.gaf_cosdist(x, y, ws)
+        assert abs(float(d.item()) - want) < 1e-6
+    a = torch.zeros(10_001, device="cuda"); a[:5000] = 1.0
+    b = torch.zeros(10_001, device="cuda"); b[5000:] = 2.0
+    d, _ = gaf.gaf_cosdist(a, b, ws)
+    assert float(d.item()) == 1.0
+    # zero-norm convention: distance 1 and a status bit
+    d, _ = gaf.gaf_cosdist(a, torch.zeros_like(a), ws)
+    assert float(d.item()) == 1.0 and gaf.gaf_read_status(ws) == gaf.GAF_STATUS_ZERO_NORM
+
+
+# ------------------------------------------------------------ Algorithm 1 ----
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_filter_small_shapes_every_tail(ws, schedule, dtype):
+    """K = 1, 2, 3, 5 and every D mod 8 (and D below one vector), several thresholds."""
+    for K in (1, 2, 3, 5):
+        for D in (0, 1, 3, 7, 8, 9, 15, 16, 17, 31, 33, 100, 257, 4096, 4099, 8200 + K):
+            w = _mix(K, D, dtype, seed=K * 1000 + D)
+            for tau in (0.5, 0.97, 1.2):
+                status = None if D == 0 else 0
+                check_filter(w.grads, tau, ws, schedule=schedule, expect_status=status)
+
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_filter_several_tiles_ragged(ws, schedule, dtype):
+    """Sizes that span several tiles per CTA, with a ragged tail, all accept patterns."""
+    D = 148 * 4096 * 3 + 148 * 1000 + 5
+    w = _mix(6, D, dtype, seed=42, rho=[0.8, 0.7, -0.6, 0.5, 0.0, 0.6])
+    seen = set()
+    for tau in (0.2, 0.6, 0.97, 1.5):
+        r = check_filter(w.grads, tau, ws, schedule=schedule)
+        seen.add(tuple(r["mask"]))
+        assert r["dist_err"] < 1e-6
+    assert len(seen) >= 3
+
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+def test_filter_order_and_special_thresholds(ws, schedule):
+    w = _mix(5, 50_001, "f32", seed=3, rho=[0.9, 0.8, 0.0, 0.7, -0.5])
+    for order in (None, [4, 3, 2, 1, 0], [2, 0, 1, 3, 4], [1, 4, 0, 2, 3]):
+        check_filter(w.grads, 0.9, ws, order=order, schedule=schedule)
+    # tau >= 2 admits everything: the plain mean of Eq. 2
+    r = check_filter(w.grads, 2.0, ws, schedule=schedule)
+    assert r["mask"] == [1] * 5 and r["count"] == 5
+    macro, *_ = gaf.gaf_filter_accumulate(w.grads, 2.0, ws, schedule=schedule)
+    mean = torch.stack([g.double() for g in w.grads]).mean(0)
+    assert float((macro.double() - mean).norm() / mean.norm()) < 1e-6
+    # a threshold nothing meets keeps only the seed, bit for bit
+    for order in (None, [3, 1, 0, 2, 4]):
+        r = check_filter(w.grads, -1.0, ws, order=order, schedule=schedule)
+        s = 0 if order is None else order[0]
+        assert r["count"] == 1 and r["mask"] == [1 if i == s else 0 for i in range(5)]
+        macro, *_ = gaf.gaf_filter_accumulate(w.grads, -1.0, ws, order=order, schedule=schedule)
+        assert torch.equal(macro, w.grads[s])
+
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+def test_filter_degenerate_inputs(ws, schedule):
+    D = 20_011
+    g = torch.randn(D, device="cuda") * 1e-3
+    z = torch.zeros(D, device="cuda")
+    # identical and opposite gradients
+    r = check_filter([g, g.clone(), -g], 0.97, ws, schedule=schedule)
+    assert r["mask"] == [1, 1, 0] and abs(r["dist"][1]) < 1e-6 and abs(r["dist"][2] - 2.0) < 1e-6
+    # inclusive threshold: exactly orthogonal integer vectors, tau = 1
+    a = torch.zeros(D, device="cuda"); a[: D // 2] = 3.0
+    b = torch.zeros(D, device="cuda"); b[D // 2:] = -2.0
+    r = check_filter([a, b], 1.0, ws, schedule=schedule)
+    assert r["dist"][1] == 1.0 and r["mask"] == [1, 1]
+    r = check_filter([a, b], math.nextafter(1.0, 0.0), ws, schedule=schedule)
+    assert r["mask"] == [1, 0]
+    # zero-norm convention (distance 1) raises a status bit, on either side of the pair
+    r = check_filter([g, z, g.clone()], 0.97, ws, schedule=schedule,
+                     expect_status=gaf.GAF_STATUS_ZERO_NORM)
+    assert r["mask"] == [1, 0, 1] and r["dist"][1] == 1.0
+    r = check_filter([z, g], 1.0, ws, schedule=schedule, expect_status=gaf.GAF_STATUS_ZERO_NORM)
+    assert r["mask"] == [1, 1]
+    # a NaN makes the distance NaN, which is rejected
+    bad = g.clone(); bad[17] = float("nan")
+    r = check_filter([g, bad, g.clone()], 1.5, ws, schedule=schedule,
+                     expect_status=gaf.GAF_STATUS_NONFINITE)
+    assert r["mask"] == [1, 0, 1] and math.isnan(r["dist"][1])
+    # wide dynamic range across the vector (a few large tensors dominate the sums)
+    scale = torch.ones(D, device="cuda"); scale[:100] = 1e4; scale[100:5000] = 1e-4
+    gs = [(torch.randn(D, device="cuda") + 0.5) * scale for _ in range(4)]
+    check_filter(gs, 0.97, ws, schedule=schedule)
+
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+def test_filter_maximum_k(ws, schedule):
+    K = gaf.binding.GAF_MAX_K
+    w = _mix(K, 10_007, "bf16", seed=64)
+    r = check_filter(w.grads, 0.97, ws, schedule=schedule)
+    assert 1 < r["count"] < K
+
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+def test_filter_bitwise_reproducible_and_workspace_reusable(ws, schedule):
+    """Fixed-order reductions: two runs agree bit for bit; the workspace needs no
+    re-initialisation between calls."""
+    w = _mix(4, 3_000_017, "f32", seed=9, rho=[0.8, 0.6, -0.2, 0.7])
+    outs = []
+    for _ in range(3):
+        macro, mask, dist, count = gaf.gaf_filter_accumulate(w.grads, 0.8, ws, schedule=schedule)
+        outs.append((macro.clone(), mask.clone(), dist.clone(), count.clone()))
+    for o in outs[1:]:
+        for x, y in zip(outs[0], o):
+            assert torch.equal(x, y)
+
+
+def test_schedules_agree(ws):
+    w = _mix(5, 2_000_003, "bf16", seed=12)
+    a = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_STEPWISE)
+    a = [t.clone() for t in a]
+    b = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_PERSISTENT)
+    assert torch.equal(a[1], b[1]) and torch.equal(a[3], b[3])
+    assert float((a[2] - b[2]).abs().max()) < 1e-6
+    assert torch.equal(a[0], b[0])       # element arithmetic is identical in both schedules
+
+
+def test_filter_host_entry_point(ws):
+    w = _mix(4, 100_003, "f32", seed=5, rho=[0.8, 0.6, -0.2, 0.7])
+    host = [g.cpu().pin_memory() for g in w.grads]
+    K, D = 4, 100_003
+    staging = torch.empty(gaf.gaf_host_staging_bytes(K, D, gaf.GAF_F32), dtype=torch.uint8, device="cuda")
+    macro_h = torch.empty(D, dtype=torch.float32).pin_memory()
+    mask_h = torch.empty(K, dtype=torch.uint8).pin_memory()
+    dist_h = torch.empty(K, dtype=torch.float32).pin_memory()
+    count_h = torch.empty(1, dtype=torch.int32).pin_memory()
+    gaf.gaf_filter_accumulate_host(host, 0.8, staging, ws, macro_h, mask_h, dist_h, count_h)
+    macro, mask, dist, count = gaf.gaf_filter_accumulate(w.grads, 0.8, ws)
+    assert torch.equal(macro.cpu(), macro_h) and torch.equal(mask.cpu(), mask_h)
+    assert torch.equal(dist.cpu(), dist_h) and int(count.item()) == int(count_h.item())
+
+
+# ------------------------------------------------- the named configurations --
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+def test_config1(ws, schedule):
+    w = workloads.config(1, device="cuda")
+    r = check_filter(w.grads, w.taus[0], ws, schedule=schedule)
+    assert r["mask"] == [1, 1, 0, 0] and r["count"] == 2       # closed form of the mixture model
+
+
+@pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
+def test_config2_resnet18_layout(ws, schedule):
+    w = workloads.config(2, device="cuda")
+    np_grads = [workloads.as_numpy_bits(g) for g in w.grads]
+    for tau in w.taus:
+        check_filter(w.grads, tau, ws, schedule=schedule, np_grads=np_grads)
+
+
+@pytest.mark.slow
+def test_config4_gpt2_small_sized(ws):
+    w = workloads.config(4, device="cuda")
+    np_grads = [workloads.as_numpy_bits(g) for g in w.grads]
+    for schedule in SCHEDULES:
+        r = check_filter(w.grads, w.taus[0], ws, schedule=schedule, np_grads=np_grads)
+        assert 1 <= r["count"] <= 8
+
+
+@pytest.mark.slow
+def test_config5_billion_bf16(ws):
+    """Full size: 8 x 1e9 bf16 (16 GB of gradients), 64-bit offsets, both schedules."""
+    free, _ = torch.cuda.mem_get_info()
+    assert free > 24 << 30, "configuration 5 needs about 21 GB of device memory"
+    w = workloads.config(5, device="cuda")
+    np_grads = [workloads.as_numpy_bits(g) for g in w.grads]
+    for schedule in SCHEDULES:
+        check_filter(w.grads, w.taus[0], ws, schedule=schedule, np_grads=np_grads)
+
+
+# ---------------------------------------------------------- pairwise matrix --
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_pairwise_small(ws, dtype):
+    for K in (1, 2, 3, 8, 9, 17, 32, 33):
+        for D in (0, 1, 5, 64, 1001, 40_003):
+            if K > 9 and D > 1001:
+                continue
+            w = _mix(K, D, dtype, seed=K * 77 + D)
+            check_pairwise(w.grads, ws)
+    w = _mix(12, 3_000_001, dtype, seed=1)
+    check_pairwise(w.grads, ws)
+
+
+def test_pairwise_zero_norm_row(ws):
+    w = _mix(4, 5001, "f32", seed=2)
+    w.grads[2].zero_()
+    check_pairwise(w.grads, ws)
+    dist, _ = gaf.gaf_pairwise_cosdist(w.grads, ws)
+    assert bool((dist[2] == 1.0).all()) and bool((dist[:, 2] == 1.0).all())
+
+
+def test_config3_pairwise(ws):
+    w = workloads.config(3, device="cuda")
+    check_pairwise(w.grads, ws)
+    dist, _ = gaf.gaf_pairwise_cosdist(w.grads, ws)
+    rho = np.array(w.rho)
+    want = 1.0 - np.sign(rho)[:, None] * np.sign(rho)[None, :] * np.sqrt(np.abs(np.outer(rho, rho)))
+    np.fill_diagonal(want, 0.0)
+    assert float(np.max(np.abs(dist.cpu().numpy() - want))) < 5e-3      # closed form of the mixture
