@@ -20,7 +20,8 @@
  *     void*; NULL = the legacy default stream) and never synchronises, except
  *     gaf_read_status and the *_host convenience call, which say so.
  *   - Gradient buffers are read-only.  Every device pointer must be 16-byte
- *     aligned (else GAF_ERR_ALIGN).  D need not be a multiple of anything.
+ *     aligned (else GAF_ERR_ALIGN).  D need not be a multiple of anything; with
+ *     D == 0 the element buffers may be NULL.
  *   - dtype: GAF_F32 = IEEE binary32, GAF_BF16 = bfloat16.  All arithmetic on
  *     elements is binary32; sums are carried in binary64 from the thread level
  *     up and reduced in a fixed order, so results are bitwise reproducible on

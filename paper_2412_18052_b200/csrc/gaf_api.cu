@@ -92,7 +92,7 @@ int check_grads(const void *const *grads, int K, int64_t D, int dtype) {
     if (!grads || K < 1 || K > GAF_MAX_K || D < 0) return GAF_ERR_ARG;
     if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
     for (int i = 0; i < K; ++i) {
-        if (!grads[i]) return GAF_ERR_ARG;
+        if (!grads[i] && D > 0) return GAF_ERR_ARG;       // an empty buffer may be NULL
         if (!aligned16(grads[i])) return GAF_ERR_ALIGN;
     }
     return GAF_OK;
@@ -136,7 +136,7 @@ int gaf_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_strea
 int gaf_cosdist(const void *x, const void *y, int64_t D, int dtype, float *dist_out,
                 double *stats_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     g_launches = 0;
-    if (!x || !y || !dist_out || D < 0) return GAF_ERR_ARG;
+    if (((!x || !y) && D > 0) || !dist_out || D < 0) return GAF_ERR_ARG;
     if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
     if (!aligned16(x) || !aligned16(y)) return GAF_ERR_ALIGN;
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
@@ -159,7 +159,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
                           size_t workspace_bytes, int schedule, void *cuda_stream) {
     g_launches = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
-    if (!macro_out || !mask_out || !count_out) return GAF_ERR_ARG;
+    if ((!macro_out && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
     if (schedule != GAF_SCHED_AUTO && schedule != GAF_SCHED_STEPWISE && schedule != GAF_SCHED_PERSISTENT)
         return GAF_ERR_ARG;
     if (tau != tau) return GAF_ERR_ARG;
@@ -230,8 +230,8 @@ int gaf_filter_accumulate_host(const void *const *grads_host, int K, int64_t D, 
     g_launches = 0;
     size_t need = 0;
     if (int rc = gaf_host_staging_bytes(K, D, dtype, &need)) return rc;
-    if (!grads_host || !macro_out_host || !mask_out_host || !count_out_host) return GAF_ERR_ARG;
-    for (int i = 0; i < K; ++i) if (!grads_host[i]) return GAF_ERR_ARG;
+    if (!grads_host || (!macro_out_host && D > 0) || !mask_out_host || !count_out_host) return GAF_ERR_ARG;
+    for (int i = 0; i < K; ++i) if (!grads_host[i] && D > 0) return GAF_ERR_ARG;
     if (int rc = check_workspace(staging, staging_bytes, need)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     auto *base = static_cast<unsigned char *>(staging);
