@@ -56,7 +56,8 @@ enum {
     GAF_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
     GAF_ERR_CUDA = 5,           /* a CUDA runtime call failed (launch, copy) */
     GAF_ERR_TIMEOUT = 6,        /* a bounded device-side wait ran out (see gaf_read_status) */
-    GAF_ERR_UNSUPPORTED = 7     /* the requested schedule cannot run on this device */
+    GAF_ERR_UNSUPPORTED = 7,    /* the requested schedule cannot run on this device */
+    GAF_ERR_TOO_LARGE = 8       /* size beyond the fixed limit of gaf_cosdist_static */
 };
 
 /* How gaf_filter_accumulate walks the K-1 sequential decisions of Algorithm 1.
@@ -179,6 +180,44 @@ int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype,
  * GAF_ERR_TIMEOUT if the timeout bit is set, else GAF_OK.
  */
 int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out);
+
+/*
+ * gaf_cosdist for callers that cannot allocate device memory.  (The paper has no
+ * counterpart of this entry point: it exists for integration reasons only.)
+ *
+ * Every other call here needs a workspace that the caller allocated.  Some
+ * callers cannot provide one: code that runs inside another framework's memory
+ * pool with allocation disabled, a plug-in called at a point where cudaMalloc
+ * would stall the whole device, a host program that is not allowed to touch the
+ * allocator after start-up.  This variant computes the same D_c(x, y) of Eq. 4
+ * with the same kernel, but keeps its scratch memory (one ticket, one status
+ * word, 512 per-CTA partial triples: 12,544 bytes) in a fixed array inside the
+ * library's device image.  It calls no cudaMalloc / cudaFree and no allocating
+ * library routine.
+ *
+ *   x, y        device, D elements of `dtype`, 16-byte aligned
+ *   D           0 .. GAF_STATIC_MAX_D; larger D returns GAF_ERR_TOO_LARGE
+ *               ("size beyond the fixed limit ...") and launches nothing
+ *   dist_out    device, 1 float;  stats_out  device, 3 doubles or NULL
+ *
+ * Things to know:
+ *   - Every GPU on which the library is loaded holds the array until the
+ *     process exits.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and remembers it.  Make
+ *     that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents;
+ *     each call clears the words that must start at zero (an asynchronous
+ *     16-word memset on the stream ahead of the kernel).  Two calls that can
+ *     overlap on the GPU (different streams without ordering, or two host
+ *     threads on one device) race on it: order them.
+ *   - The status word is not readable through gaf_read_status (that call takes a
+ *     workspace); the zero-norm convention still applies (distance 1).
+ *   - Asynchronous on `cuda_stream`, like gaf_cosdist.
+ */
+#define GAF_STATIC_MAX_D ((int64_t)1 << 31)
+int gaf_cosdist_static(const void *x, const void *y, int64_t D, int dtype,
+                       float *dist_out, double *stats_out, void *cuda_stream);
 
 /* Number of kernel launches the most recent gaf_* call of this thread issued
  * (host-side counter, for benchmarks). */

@@ -23,7 +23,7 @@ _lib = None
 EXPORTS = [
     "gaf_error_string", "gaf_workspace_bytes", "gaf_workspace_init", "gaf_cosdist",
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
-    "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count",
+    "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
 ]
 
 
@@ -56,6 +56,7 @@ def lib() -> ctypes.CDLL:
         L.gaf_pairwise_cosdist.argtypes = [vp, i32, i64, i32, vp, vp, vp, sz, vp]
         L.gaf_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.gaf_last_launch_count.argtypes = []
+        L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         for name in EXPORTS:
             if name != "gaf_error_string":
                 getattr(L, name).restype = i32
@@ -128,6 +129,19 @@ def gaf_cosdist(x: torch.Tensor, y: torch.Tensor, workspace: torch.Tensor,
                              dist_out.data_ptr(), stats_out.data_ptr(),
                              workspace.data_ptr(), workspace.numel(), _stream()), "gaf_cosdist")
     return dist_out, stats_out
+
+
+def gaf_cosdist_static(x: torch.Tensor, y: torch.Tensor, dist_out: torch.Tensor,
+                       stats_out: Optional[torch.Tensor] = None) -> None:
+    """Eq. 4 between two device tensors without any workspace: for callers that
+    may not allocate device memory (the scratch is a fixed array inside the
+    library).  The outputs are the caller's tensors; nothing is allocated here
+    either.  Calls must not overlap on the GPU; D is limited to 2**31."""
+    assert x.numel() == y.numel() and x.dtype == y.dtype
+    _check(lib().gaf_cosdist_static(x.data_ptr(), y.data_ptr(), x.numel(), _dtype_code(x),
+                                    dist_out.data_ptr(),
+                                    None if stats_out is None else stats_out.data_ptr(), _stream()),
+           "gaf_cosdist_static")
 
 
 def gaf_filter_accumulate(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,

@@ -112,6 +112,7 @@ const char *gaf_error_string(int code) {
         case GAF_ERR_CUDA: return "CUDA runtime error";
         case GAF_ERR_TIMEOUT: return "device-side wait timed out";
         case GAF_ERR_UNSUPPORTED: return "schedule not supported on this device";
+        case GAF_ERR_TOO_LARGE: return "size beyond the fixed limit of the no-allocation entry point";
         default: return "unknown error code";
     }
 }
