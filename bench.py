@@ -45,7 +45,7 @@ def parse_args():
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 4, 5],
                     help="named configuration (2 is the one the metric is quoted on)")
     ap.add_argument("--tau", type=float, default=0.97)
-    ap.add_argument("--schedule", type=int, default=0, help="0 auto, 1 stepwise, 2 persistent")
+    ap.add_argument("--schedule", type=int, default=0, help="0 auto, 1 stepwise, 2 persistent, 3 resident")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -318,7 +318,7 @@ def run_ours(args):
                             f"shared+private Gaussian mixture" +
                             (" with ResNet18 per-tensor scales" if cfg == 2 else ""),
                 "K": K, "D": D, "input_dtype": w0.dtype, "tau": args.tau,
-                "schedule": {0: "auto", 1: "stepwise", 2: "persistent"}[args.schedule],
+                "schedule": {0: "auto", 1: "stepwise", 2: "persistent", 3: "resident"}[args.schedule],
                 "parallelism": "replicas only (the path does not shard)" if world > 1 else "1 GPU",
                 "l2": f"{n_sets} rotating input sets of {grad_bytes / 1e6:.0f} MB each (inputs of a step "
                       f"exceed the 126 MB L2 and were last touched {n_sets - 1} steps earlier)"

@@ -66,8 +66,11 @@ enum {
 enum {
     GAF_SCHED_AUTO = 0,         /* the library picks */
     GAF_SCHED_STEPWISE = 1,     /* one launch per step; decisions stay on the device */
-    GAF_SCHED_PERSISTENT = 2    /* one cooperative launch; bulk-async shared-memory
+    GAF_SCHED_PERSISTENT = 2,   /* one cooperative launch; bulk-async shared-memory
                                    pipeline that keeps prefetching across decisions */
+    GAF_SCHED_RESIDENT = 3      /* one cooperative launch; the running sum stays in
+                                   registers and shared memory between passes (spills to
+                                   macro_out only when D exceeds the on-chip capacity) */
 };
 
 /* Bits of the device status word. */

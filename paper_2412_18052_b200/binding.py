@@ -13,7 +13,7 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 GAF_F32, GAF_BF16 = 0, 1
-GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_PERSISTENT = 0, 1, 2
+GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_PERSISTENT, GAF_SCHED_RESIDENT = 0, 1, 2, 3
 GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT = 1, 2, 4
 GAF_MAX_K = 64
 

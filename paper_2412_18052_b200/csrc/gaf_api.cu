@@ -9,6 +9,7 @@
 #include "gaf_device.cuh"
 #include "gaf_pairwise.cuh"
 #include "gaf_persistent.cuh"
+#include "gaf_resident.cuh"
 #include "gaf_stepwise.cuh"
 
 namespace {
@@ -161,7 +162,8 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     g_launches = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if ((!macro_out && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
-    if (schedule != GAF_SCHED_AUTO && schedule != GAF_SCHED_STEPWISE && schedule != GAF_SCHED_PERSISTENT)
+    if (schedule != GAF_SCHED_AUTO && schedule != GAF_SCHED_STEPWISE && schedule != GAF_SCHED_PERSISTENT &&
+        schedule != GAF_SCHED_RESIDENT)
         return GAF_ERR_ARG;
     if (tau != tau) return GAF_ERR_ARG;
     if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
@@ -192,8 +194,21 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
     if (schedule == GAF_SCHED_AUTO) {
-        schedule = (K >= 2 && persistent_supported(di.coop, di.smem_optin)) ? GAF_SCHED_PERSISTENT
-                                                                          : GAF_SCHED_STEPWISE;
+        // on-chip running sum whenever it fits; otherwise one launch per step
+        const bool fits = D <= resident_capacity(di.sms, di.smem_optin);
+        schedule = (K >= 2 && di.coop && fits) ? GAF_SCHED_RESIDENT : GAF_SCHED_STEPWISE;
+    }
+    if (schedule == GAF_SCHED_RESIDENT) {
+        if (!di.coop) return GAF_ERR_UNSUPPORTED;
+        if (K >= 2) {
+            int rc = dtype == GAF_F32
+                ? launch_resident<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
+                                         ctl, partials, di.sms, di.smem_optin, st)
+                : launch_resident<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
+                                                 count_out, ctl, partials, di.sms, di.smem_optin, st);
+            if (rc == GAF_OK) ++g_launches;
+            return rc;
+        }
     }
     if (schedule == GAF_SCHED_PERSISTENT) {
         if (!persistent_supported(di.coop, di.smem_optin)) return GAF_ERR_UNSUPPORTED;

@@ -33,8 +33,8 @@ def test_every_declared_symbol_is_exported(L):
 
 
 def test_error_strings(L):
-    seen = {L.gaf_error_string(c) for c in range(0, 8)}
-    assert len(seen) == 8 and b"unknown error code" not in seen
+    seen = {L.gaf_error_string(c) for c in range(0, 9)}
+    assert len(seen) == 9 and b"unknown error code" not in seen
     assert L.gaf_error_string(1234) == b"unknown error code"
 
 

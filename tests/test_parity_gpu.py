@@ -12,8 +12,8 @@ from parity import check_cosdist, check_filter, check_pairwise
 
 pytestmark = pytest.mark.gpu
 
-SCHEDULES = [gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_PERSISTENT]
-SCHED_IDS = ["stepwise", "persistent"]
+SCHEDULES = [gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_PERSISTENT, gaf.GAF_SCHED_RESIDENT]
+SCHED_IDS = ["stepwise", "persistent", "resident"]
 DTYPES = ["f32", "bf16"]
 
 
@@ -166,10 +166,11 @@ def test_schedules_agree(ws):
     w = _mix(5, 2_000_003, "bf16", seed=12)
     a = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_STEPWISE)
     a = [t.clone() for t in a]
-    b = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_PERSISTENT)
-    assert torch.equal(a[1], b[1]) and torch.equal(a[3], b[3])
-    assert float((a[2] - b[2]).abs().max()) < 1e-6
-    assert torch.equal(a[0], b[0])       # element arithmetic is identical in both schedules
+    for other in (gaf.GAF_SCHED_PERSISTENT, gaf.GAF_SCHED_RESIDENT, gaf.GAF_SCHED_AUTO):
+        b = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=other)
+        assert torch.equal(a[1], b[1]) and torch.equal(a[3], b[3])
+        assert float((a[2] - b[2]).abs().max()) < 1e-6
+        assert torch.equal(a[0], b[0])       # element arithmetic is identical in every schedule
 
 
 def test_filter_host_entry_point(ws):
