@@ -55,29 +55,33 @@ enum {
     GAF_ERR_ALIAS = 3,          /* macro_out overlaps an input gradient */
     GAF_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
     GAF_ERR_CUDA = 5,           /* a CUDA runtime call failed (launch, copy) */
-    GAF_ERR_TIMEOUT = 6,        /* a bounded device-side wait ran out (see gaf_read_status) */
+    GAF_ERR_RESERVED = 6,       /* not used */
     GAF_ERR_UNSUPPORTED = 7,    /* the requested schedule cannot run on this device */
     GAF_ERR_TOO_LARGE = 8       /* size beyond the fixed limit of gaf_cosdist_static */
 };
 
 /* How gaf_filter_accumulate walks the K-1 sequential decisions of Algorithm 1.
- * All schedules compute the same values in the same order of operations per
- * element; they differ in launch structure only. */
+ * Both schedules produce the same mask and a bit-identical macro-gradient (the
+ * accepted gradients are always added in processing order in binary32); they
+ * differ in launch structure and in how many bytes cross HBM. */
 enum {
-    GAF_SCHED_AUTO = 0,         /* the library picks */
-    GAF_SCHED_STEPWISE = 1,     /* one launch per step; decisions stay on the device */
-    GAF_SCHED_PERSISTENT = 2,   /* one cooperative launch; bulk-async shared-memory
-                                   pipeline that keeps prefetching across decisions */
-    GAF_SCHED_RESIDENT = 3      /* one cooperative launch; the running sum stays in
-                                   registers and shared memory between passes (spills to
-                                   macro_out only when D exceeds the on-chip capacity) */
+    GAF_SCHED_AUTO = 0,         /* the library picks (Gram-first for K <= 8) */
+    GAF_SCHED_STEPWISE = 1,     /* streaming: one launch per step; each launch adds the
+                                   gradient accepted at step t to the running sum and, in
+                                   the same pass, takes the three dot products of the
+                                   updated sum with the candidate of step t+1; decisions
+                                   stay on the device */
+    GAF_SCHED_GRAM = 2          /* Gram-first: every gradient is read once to build the
+                                   K x K Gram matrix, the K-1 decisions are taken on it (dot
+                                   products are bilinear), then the accepted gradients are
+                                   read once more to write g/c.  The distances agree with
+                                   the stepwise schedule to rounding. */
 };
 
 /* Bits of the device status word. */
 enum {
     GAF_STATUS_ZERO_NORM = 1,   /* some tested pair had a zero norm (distance set to 1) */
-    GAF_STATUS_NONFINITE = 2,   /* some sum was NaN or Inf */
-    GAF_STATUS_TIMEOUT = 4      /* a bounded wait expired; outputs are not valid */
+    GAF_STATUS_NONFINITE = 2    /* some sum was NaN or Inf */
 };
 
 /* Human-readable name of a return code.  Host only; never NULL. */
@@ -92,9 +96,8 @@ int gaf_workspace_bytes(int K, int64_t D, int dtype, size_t *bytes_out);
 
 /*
  * Prepare a workspace: clears its control block (asynchronous memset on the
- * stream).  Needed once after allocation, and again after a call reported
- * GAF_STATUS_TIMEOUT; calls that finish normally leave the workspace ready for
- * the next call.  A workspace serves one call at a time: calls that share a
+ * stream).  Needed once after allocation; every call leaves the workspace ready
+ * for the next one.  A workspace serves one call at a time: calls that share a
  * workspace must be ordered on one stream.
  *   workspace        device, 256-byte aligned, >= gaf_workspace_bytes(...)
  */
@@ -179,8 +182,7 @@ int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype,
 
 /*
  * Read the device status word of the most recent call that used `workspace`.
- * SYNCHRONISES the stream.  *status_out receives GAF_STATUS_* bits.  Returns
- * GAF_ERR_TIMEOUT if the timeout bit is set, else GAF_OK.
+ * SYNCHRONISES the stream.  *status_out receives GAF_STATUS_* bits.
  */
 int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out);
 

@@ -13,8 +13,8 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 GAF_F32, GAF_BF16 = 0, 1
-GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_PERSISTENT, GAF_SCHED_RESIDENT = 0, 1, 2, 3
-GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT = 1, 2, 4
+GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_GRAM = 0, 1, 2
+GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE = 1, 2
 GAF_MAX_K = 64
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgaf.so")
@@ -216,9 +216,7 @@ def gaf_pairwise_cosdist(grads: Sequence[torch.Tensor], workspace: torch.Tensor,
 def gaf_read_status(workspace: torch.Tensor) -> int:
     """Status bits of the latest call on this workspace (synchronises the stream)."""
     out = ctypes.c_int()
-    rc = lib().gaf_read_status(workspace.data_ptr(), _stream(), ctypes.byref(out))
-    if rc not in (0, 6):
-        raise GafError(rc, "gaf_read_status")
+    _check(lib().gaf_read_status(workspace.data_ptr(), _stream(), ctypes.byref(out)), "gaf_read_status")
     return out.value
 
 

@@ -7,9 +7,8 @@
 
 #include "../../include/gaf.h"
 #include "gaf_device.cuh"
+#include "gaf_gramfilter.cuh"
 #include "gaf_pairwise.cuh"
-#include "gaf_persistent.cuh"
-#include "gaf_resident.cuh"
 #include "gaf_stepwise.cuh"
 
 namespace {
@@ -20,35 +19,19 @@ thread_local int g_launches = 0;
 
 struct DeviceInfo {
     int sms = 0;
-    int coop = 0;
-    int smem_optin = 0;
 };
 
-// Attributes of the current device (queried per call: two cheap driver lookups).
+// Attributes of the current device (queried per call: a cheap driver lookup).
 bool device_info(DeviceInfo *out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&out->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&out->coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&out->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-        return false;
     return out->sms > 0;
 }
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t elem_bytes(int dtype) { return dtype == GAF_F32 ? 4 : 2; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
-size_t pairwise_extra_bytes(int K) {
-    const int tiles = (K + kGramTile - 1) / kGramTile;
-    const size_t pairs = size_t(tiles) * (tiles + 1) / 2;
-    return pairs * kGramMaxSlices * 64 * sizeof(double) + round_up(size_t(K) * K * sizeof(double), 256);
-}
-
-int check_workspace(const void *ws, size_t have, size_t need) {
-    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || have < need) return GAF_ERR_WORKSPACE;
-    return GAF_OK;
-}
 
 // CTAs for a streaming kernel of `threads` threads that handles 8 elements per
 // thread and iteration: two per SM, fewer when D is small.
@@ -58,6 +41,119 @@ int stream_grid(int64_t D, int threads, int sms) {
     if (cap > kMaxCtas) cap = kMaxCtas;
     if (need < 1) need = 1;
     return int(need < cap ? need : cap);
+}
+
+// Layout after the per-CTA triples: Gram partials [tile pair][slice][64] doubles, the
+// Gram matrix by original index, the Gram matrix by processing step, a K x K float
+// scratch for distances nobody asked for.
+size_t gram_partials_bytes(int K) {
+    const int tiles = (K + kGramTile - 1) / kGramTile;
+    const size_t pairs = size_t(tiles) * (tiles + 1) / 2;
+    return pairs * kGramMaxSlices * 64 * sizeof(double);
+}
+size_t gram_matrix_bytes(int K) { return round_up(size_t(K) * K * sizeof(double), 256); }
+size_t pairwise_extra_bytes(int K) { return gram_partials_bytes(K) + 3 * gram_matrix_bytes(K); }
+
+// Tiled Gram matrix of K gradients (by original index) into the workspace; optional
+// distance matrix.  Two launches.
+int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, float *dist_out,
+                      double *gram_out, unsigned char *base, int sms, cudaStream_t st) {
+    GramArgs a{};
+    for (int i = 0; i < K; ++i) a.g[i] = grads[i];
+    a.K = K; a.D = D;
+    a.tiles = (K + kGramTile - 1) / kGramTile;
+    const int pairs = a.tiles * (a.tiles + 1) / 2;
+    a.partials = reinterpret_cast<double *>(base + kExtraOffset);
+    a.gram = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K));
+    a.dist_out = dist_out ? dist_out
+                          : reinterpret_cast<float *>(base + kExtraOffset + gram_partials_bytes(K) +
+                                                      2 * gram_matrix_bytes(K));
+    a.gram_out = gram_out;
+    a.ctl = reinterpret_cast<Control *>(base);
+    // D-slices: fill the machine about twice over all tile pairs, never more than there is work
+    int64_t slices = (int64_t(sms) * 2 + pairs - 1) / pairs;
+    const int64_t work = (D / 4 + kGramThreads - 1) / kGramThreads;
+    if (slices > work) slices = work;
+    if (slices > kGramMaxSlices) slices = kGramMaxSlices;
+    if (slices < 1) slices = 1;
+    a.slices = int(slices);
+    dim3 grid(a.slices, pairs);
+    if (dtype == GAF_F32) gram_tile_kernel<float><<<grid, kGramThreads, 0, st>>>(a);
+    else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
+    ++g_launches;
+    gram_finish_kernel<<<pairs, 256, 0, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+template <typename T, int KT>
+int launch_gram_small_kt(const GramSmallArgs &a, int sms, cudaStream_t st) {
+    int occ = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gram_small_kernel<T, KT>, kGsThreads, 0) !=
+        cudaSuccess || occ < 1)
+        occ = 1;
+    if (occ > 2) occ = 2;
+    int64_t grid = int64_t(sms) * occ;
+    if (grid > kGsMaxCtas) grid = kGsMaxCtas;
+    const int64_t work = (a.D / GsVec<T>::N + kGsThreads - 1) / kGsThreads;
+    if (grid > work) grid = work;
+    if (grid < 1) grid = 1;
+    gram_small_kernel<T, KT><<<int(grid), kGsThreads, 0, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+template <typename T>
+int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
+    switch (K) {
+        case 2: return launch_gram_small_kt<T, 2>(a, sms, st);
+        case 3: return launch_gram_small_kt<T, 3>(a, sms, st);
+        case 4: return launch_gram_small_kt<T, 4>(a, sms, st);
+        case 5: return launch_gram_small_kt<T, 5>(a, sms, st);
+        case 6: return launch_gram_small_kt<T, 6>(a, sms, st);
+        case 7: return launch_gram_small_kt<T, 7>(a, sms, st);
+        case 8: return launch_gram_small_kt<T, 8>(a, sms, st);
+        default: return GAF_ERR_ARG;
+    }
+}
+
+// Gram-first schedule: Gram matrix, scalar walk of Algorithm 1, masked mean.
+template <typename T>
+int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double tau, const int32_t *ord,
+                      float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
+                      unsigned char *base, int sms, cudaStream_t st) {
+    Control *ctl = reinterpret_cast<Control *>(base);
+    ReplayArgs r{};
+    r.K = K; r.tau = tau; r.mask_out = mask_out; r.dist_out = dist_out; r.count_out = count_out; r.ctl = ctl;
+    for (int t = 0; t < K; ++t) r.idx[t] = ord[t];
+    double *gram_by_index = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K));
+    double *gram_by_step = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K) +
+                                                      gram_matrix_bytes(K));
+    if (K <= kGsMaxK) {
+        GramSmallArgs a{};
+        for (int t = 0; t < K; ++t) a.g[t] = g[ord[t]];
+        a.D = D;
+        a.partials = reinterpret_cast<double *>(base + kExtraOffset);
+        a.gram = gram_by_step;
+        a.replay = r;
+        if (int rc = launch_gram_small<T>(a, K, sms, st)) return rc;
+    } else {
+        if (int rc = launch_gram_tiles(g, K, D, dtype, nullptr, nullptr, base, sms, st)) return rc;
+        gram_replay_kernel<<<1, 256, 0, st>>>(r, gram_by_index, gram_by_step);
+        ++g_launches;
+    }
+    MaskedMeanArgs m{};
+    for (int t = 0; t < K; ++t) m.g[t] = g[ord[t]];
+    m.K = K; m.D = D; m.out = macro_out; m.ctl = ctl;
+    const int grid = stream_grid(D, kMsThreads, sms);
+    masked_mean_kernel<T><<<grid, kMsThreads, 0, st>>>(m);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int check_workspace(const void *ws, size_t have, size_t need) {
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || have < need) return GAF_ERR_WORKSPACE;
+    return GAF_OK;
 }
 
 template <typename T>
@@ -111,7 +207,7 @@ const char *gaf_error_string(int code) {
         case GAF_ERR_ALIAS: return "macro_out overlaps an input gradient";
         case GAF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case GAF_ERR_CUDA: return "CUDA runtime error";
-        case GAF_ERR_TIMEOUT: return "device-side wait timed out";
+        case GAF_ERR_RESERVED: return "reserved";
         case GAF_ERR_UNSUPPORTED: return "schedule not supported on this device";
         case GAF_ERR_TOO_LARGE: return "size beyond the fixed limit of the no-allocation entry point";
         default: return "unknown error code";
@@ -162,9 +258,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     g_launches = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if ((!macro_out && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
-    if (schedule != GAF_SCHED_AUTO && schedule != GAF_SCHED_STEPWISE && schedule != GAF_SCHED_PERSISTENT &&
-        schedule != GAF_SCHED_RESIDENT)
-        return GAF_ERR_ARG;
+    if (schedule < GAF_SCHED_AUTO || schedule > GAF_SCHED_GRAM) return GAF_ERR_ARG;
     if (tau != tau) return GAF_ERR_ARG;
     if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
     int32_t ord[GAF_MAX_K];
@@ -194,33 +288,18 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
     if (schedule == GAF_SCHED_AUTO) {
-        // on-chip running sum whenever it fits; otherwise one launch per step
-        const bool fits = D <= resident_capacity(di.sms, di.smem_optin);
-        schedule = (K >= 2 && di.coop && fits) ? GAF_SCHED_RESIDENT : GAF_SCHED_STEPWISE;
+        // Gram-first moves fewer bytes whenever its one-pass Gram kernel applies
+        const bool ws_ok = workspace_bytes >= kExtraOffset + pairwise_extra_bytes(K);
+        schedule = (K >= 2 && K <= kGsMaxK && ws_ok) ? GAF_SCHED_GRAM : GAF_SCHED_STEPWISE;
     }
-    if (schedule == GAF_SCHED_RESIDENT) {
-        if (!di.coop) return GAF_ERR_UNSUPPORTED;
-        if (K >= 2) {
-            int rc = dtype == GAF_F32
-                ? launch_resident<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
-                                         ctl, partials, di.sms, di.smem_optin, st)
-                : launch_resident<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
-                                                 count_out, ctl, partials, di.sms, di.smem_optin, st);
-            if (rc == GAF_OK) ++g_launches;
+    if (schedule == GAF_SCHED_GRAM && K >= 2) {
+        if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K)))
             return rc;
-        }
-    }
-    if (schedule == GAF_SCHED_PERSISTENT) {
-        if (!persistent_supported(di.coop, di.smem_optin)) return GAF_ERR_UNSUPPORTED;
-        if (K >= 2) {
-            int rc = dtype == GAF_F32
-                ? launch_persistent<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
-                                           count_out, ctl, partials, di.sms, st)
-                : launch_persistent<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out,
-                                                   dist_out, count_out, ctl, partials, di.sms, st);
-            if (rc == GAF_OK) ++g_launches;
-            return rc;
-        }
+        return dtype == GAF_F32
+            ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
+                                       count_out, base, di.sms, st)
+            : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
+                                               count_out, base, di.sms, st);
     }
     return dtype == GAF_F32
         ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
@@ -288,31 +367,8 @@ int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype, 
     DeviceInfo di;
     if (!device_info(&di)) return GAF_ERR_CUDA;
     auto *base = static_cast<unsigned char *>(workspace);
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    GramArgs a{};
-    for (int i = 0; i < K; ++i) a.g[i] = grads[i];
-    a.K = K; a.D = D;
-    a.tiles = (K + kGramTile - 1) / kGramTile;
-    const int pairs = a.tiles * (a.tiles + 1) / 2;
-    a.partials = reinterpret_cast<double *>(base + kExtraOffset);
-    a.gram = reinterpret_cast<double *>(base + kExtraOffset +
-                                        size_t(pairs) * kGramMaxSlices * 64 * sizeof(double));
-    a.dist_out = dist_out; a.gram_out = gram_out;
-    a.ctl = reinterpret_cast<Control *>(base);
-    // D-slices: fill the machine about twice over all tile pairs, never more than there is work
-    int64_t slices = (int64_t(di.sms) * 2 + pairs - 1) / pairs;
-    const int64_t work = (D / 4 + kGramThreads - 1) / kGramThreads;
-    if (slices > work) slices = work;
-    if (slices > kGramMaxSlices) slices = kGramMaxSlices;
-    if (slices < 1) slices = 1;
-    a.slices = int(slices);
-    dim3 grid(a.slices, pairs);
-    if (dtype == GAF_F32) gram_tile_kernel<float><<<grid, kGramThreads, 0, st>>>(a);
-    else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
-    ++g_launches;
-    gram_finish_kernel<<<pairs, 256, 0, st>>>(a);
-    ++g_launches;
-    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+    return launch_gram_tiles(grads, K, D, dtype, dist_out, gram_out, base, di.sms,
+                             static_cast<cudaStream_t>(cuda_stream));
 }
 
 int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out) {
@@ -324,7 +380,7 @@ int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out) {
         return GAF_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return GAF_ERR_CUDA;
     *status_out = status;
-    return (status & GAF_STATUS_TIMEOUT) ? GAF_ERR_TIMEOUT : GAF_OK;
+    return GAF_OK;
 }
 
 }  // extern "C"

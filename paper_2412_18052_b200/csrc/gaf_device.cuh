@@ -17,11 +17,12 @@ constexpr int kOct = 8;                 // elements handled per inner step
 // Control block at the start of the caller's workspace.
 struct Control {
     unsigned int ticket;                // last-block election, wraps to 0 by itself
-    unsigned int barrier;               // arrivals at the grid barrier (persistent schedule)
-    unsigned int exit_ticket;           // persistent schedule: resets `barrier` at the end
+    unsigned int reserved0;
+    unsigned int reserved1;
     int status;                         // GAF_STATUS_* bits of the latest call
     int count;                          // running c of Algorithm 1
-    int pad[3];
+    int pad;
+    unsigned long long accept_bits;     // Gram-first schedule: bit t set = step t accepted
     int decision[GAF_MAX_K];            // by step t: 1 accept, 0 reject
     double sums[GAF_MAX_K][3];          // by step t: {g_i.g, |g|^2, |g_i|^2}
 };

@@ -1,0 +1,274 @@
+// Gram-first schedule of Algorithm 1.
+//
+// The test of step t needs <g_i, g>, |g|^2 and |g_i|^2 where g is the sum of the
+// gradients accepted so far.  Dot products are bilinear, so all of them follow from
+// the K x K Gram matrix G_ij = <g_i, g_j> of the raw micro-gradients:
+//     <g_i, sum_A g_j> = sum_{j in A} G_ji,     |sum_A g_j|^2 = sum_{j,l in A} G_jl.
+// The schedule therefore reads every gradient ONCE to build G (binary64 sums), walks
+// the K-1 sequential decisions of Algorithm 1 on K^2 scalars in a single thread, and
+// then reads only the accepted gradients once more to write g/c (Eq. 5):
+// ((K + c) b + 4) D bytes instead of one pass over the running sum per step, and no
+// grid-wide serialisation per step.  The accepted gradients are added in processing
+// order in binary32, so the macro-gradient is bit-identical to the streaming
+// schedules'; the distances differ from theirs only by rounding (the running sum is
+// never rounded to binary32 here).
+#pragma once
+
+#include "gaf_device.cuh"
+
+namespace gaf {
+
+constexpr int kGsThreads = 512;
+constexpr int kGsMaxK = 8;                  // gradients the one-pass register-tiled Gram handles
+constexpr int kGsMaxCtas = 296;
+constexpr int kGsFlushEvery = 16;           // iterations between binary64 flushes
+constexpr int kMsThreads = 512;
+
+struct ReplayArgs {
+    int K;
+    double tau;
+    int idx[GAF_MAX_K];                     // original index of the gradient processed at step t
+    uint8_t *mask_out;
+    float *dist_out;                        // may be null
+    int32_t *count_out;
+    Control *ctl;
+};
+
+// Algorithm 1 on the Gram matrix (indexed by processing step): one thread.
+// gram is K x K row-major in binary64.
+__device__ __forceinline__ void replay_on_gram(const ReplayArgs &r, const volatile double *gram) {
+    const int K = r.K;
+    Control *c = r.ctl;
+    int status = 0, count = 1;
+    unsigned long long bits = 1ull;         // bit t set = step t accepted (step 0 is the seed)
+    double na = gram[0];                    // |g|^2 of the running sum
+    c->decision[0] = 1;
+    r.mask_out[r.idx[0]] = 1;
+    if (r.dist_out) r.dist_out[r.idx[0]] = 0.0f;
+    for (int t = 1; t < K; ++t) {
+        double p = 0.0;                     // <g_t, running sum>
+        for (int u = 0; u < t; ++u)
+            if ((bits >> u) & 1ull) p += gram[(size_t)u * K + t];
+        const double ng = gram[(size_t)t * K + t];
+        const double d = cosine_distance(p, na, ng, &status);
+        const int accept = (d <= r.tau) ? 1 : 0;
+        c->decision[t] = accept;
+        c->sums[t][0] = p; c->sums[t][1] = na; c->sums[t][2] = ng;
+        r.mask_out[r.idx[t]] = (uint8_t)accept;
+        if (r.dist_out) r.dist_out[r.idx[t]] = (float)d;
+        if (accept) {
+            bits |= 1ull << t;
+            na = na + 2.0 * p + ng;         // |g + g_t|^2
+            ++count;
+        }
+    }
+    c->accept_bits = bits;
+    c->count = count;
+    c->status = status;
+    *r.count_out = count;
+    __threadfence();
+}
+
+// ------------------------------------------------ one-pass Gram for K <= 8 ----
+
+struct GramSmallArgs {
+    const void *g[kGsMaxK];                 // processing order
+    int64_t D;
+    double *partials;                       // [cta][64]
+    double *gram;                           // [K][K]
+    ReplayArgs replay;
+};
+
+template <typename T> struct GsVec;         // one 16-byte load per gradient and iteration
+template <> struct GsVec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const float *base, int64_t e, float (&v)[4]) {
+        float4 a = __ldcs(reinterpret_cast<const float4 *>(base + e));
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    }
+};
+template <> struct GsVec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *base, int64_t e, float (&v)[8]) {
+        uint4 r = __ldcs(reinterpret_cast<const uint4 *>(base + e));
+        unsigned int w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[2 * k] = bf16_bits_to_float(w[k] & 0xFFFFu);
+            v[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        }
+    }
+};
+
+template <typename T, int KT>
+__global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_constant__ GramSmallArgs a) {
+    constexpr int NP = KT * (KT + 1) / 2;   // upper triangle
+    constexpr int N = GsVec<T>::N;
+    __shared__ double sacc[kGsThreads / 32][NP];
+    __shared__ bool is_last;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
+    __syncwarp();
+
+    const T *row[KT];
+#pragma unroll
+    for (int r = 0; r < KT; ++r) row[r] = static_cast<const T *>(a.g[r]);
+
+    float acc[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) acc[p] = 0.0f;
+
+    auto flush = [&]() {
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            float v = acc[p];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
+            if (lane == 0) sacc[warp][p] += (double)v;
+            acc[p] = 0.0f;
+        }
+    };
+
+    const int64_t n_vec = a.D / N;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int since_flush = 0;
+    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n_vec; q += stride) {
+        float x[KT][N];
+#pragma unroll
+        for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], q * N, x[r]);
+        int p = 0;
+#pragma unroll
+        for (int r = 0; r < KT; ++r)
+#pragma unroll
+            for (int c = r; c < KT; ++c, ++p) {
+                float s = acc[p];
+#pragma unroll
+                for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
+                acc[p] = s;
+            }
+        if (++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+    }
+    // ragged tail (D mod N elements), first CTA
+    const int64_t tail0 = n_vec * N;
+    if (blockIdx.x == 0 && tail0 + threadIdx.x < a.D) {
+        const int64_t e = tail0 + threadIdx.x;
+        float x[KT];
+#pragma unroll
+        for (int r = 0; r < KT; ++r) x[r] = load1<T>(row[r], e);
+        int p = 0;
+#pragma unroll
+        for (int r = 0; r < KT; ++r)
+#pragma unroll
+            for (int c = r; c < KT; ++c, ++p) acc[p] = fmaf(x[r], x[c], acc[p]);
+    }
+    flush();
+    __syncthreads();
+    if (threadIdx.x < NP) {
+        double s = 0.0;
+        for (int w = 0; w < kGsThreads / 32; ++w) s += sacc[w][threadIdx.x];
+        a.partials[(size_t)blockIdx.x * 64 + threadIdx.x] = s;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int old = atomicInc(&a.replay.ctl->ticket, gridDim.x - 1);
+        is_last = (old == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // last CTA: fixed-order totals (one warp per pair), then the scalar walk
+    const volatile double *part = a.partials;
+    for (int p = warp; p < NP; p += kGsThreads / 32) {
+        double s = 0.0;
+        for (int i = lane; i < (int)gridDim.x; i += 32) s += part[(size_t)i * 64 + p];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) s += shfl_down_f64(s, d);
+        if (lane == 0) {
+            // decode p -> (r, c), r <= c
+            int r = 0, rem = p;
+            while (rem >= KT - r) { rem -= KT - r; ++r; }
+            const int c = r + rem;
+            a.gram[r * KT + c] = s;
+            a.gram[c * KT + r] = s;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) replay_on_gram(a.replay, a.gram);
+}
+
+// Scalar walk as its own launch (Gram matrix produced by the tiled pairwise kernels).
+// `perm` maps processing step -> row of `gram_by_index` (K x K by original index).
+__global__ void gram_replay_kernel(ReplayArgs r, const double *gram_by_index, double *gram_by_step) {
+    const int K = r.K;
+    for (int i = threadIdx.x; i < K * K; i += blockDim.x) {
+        const int t = i / K, u = i % K;
+        gram_by_step[i] = gram_by_index[(size_t)r.idx[t] * K + r.idx[u]];
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) replay_on_gram(r, gram_by_step);
+}
+
+// ------------------------------------------------------- masked mean (Eq. 5) --
+
+struct MaskedMeanArgs {
+    const void *g[GAF_MAX_K];               // processing order
+    int K;
+    int64_t D;
+    float *out;
+    const Control *ctl;
+};
+
+// out = (((g_0 + g_a) + g_b) + ...) / c over the accepted steps a < b < ..., binary32,
+// in processing order: the same association as the streaming schedules.
+template <typename T>
+__global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid_constant__ MaskedMeanArgs a) {
+    __shared__ const T *list[GAF_MAX_K];
+    __shared__ int n_list;
+    __shared__ float cdiv_s;
+    if (threadIdx.x == 0) {
+        const unsigned long long bits = *reinterpret_cast<const volatile unsigned long long *>(&a.ctl->accept_bits);
+        int n = 0;
+        for (int t = 0; t < a.K; ++t)
+            if ((bits >> t) & 1ull) list[n++] = static_cast<const T *>(a.g[t]);
+        n_list = n;
+        cdiv_s = (float)n;
+    }
+    __syncthreads();
+    const int n = n_list;
+    const float cdiv = cdiv_s;
+    const int64_t n_oct = a.D / kOct;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < n_oct; o += stride) {
+        const int64_t e = o * kOct;
+        float v[8];
+        load8_stream<T>(list[0], e, v);
+        for (int i = 1; i < n; i += 4) {
+            float w[4][8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i + u < n) load8_stream<T>(list[i + u], e, w[u]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i + u < n) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) v[k] += w[u][k];
+                }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = v[k] / cdiv;
+        store8(a.out, e, v, true);
+    }
+    const int64_t tail0 = n_oct * kOct;
+    if (blockIdx.x == 0 && tail0 + threadIdx.x < a.D) {
+        const int64_t e = tail0 + threadIdx.x;
+        float v = load1<T>(list[0], e);
+        for (int i = 1; i < n; ++i) v += load1<T>(list[i], e);
+        a.out[e] = v / cdiv;
+    }
+}
+
+}  // namespace gaf
