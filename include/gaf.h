@@ -81,7 +81,9 @@ enum {
 /* Bits of the device status word. */
 enum {
     GAF_STATUS_ZERO_NORM = 1,   /* some tested pair had a zero norm (distance set to 1) */
-    GAF_STATUS_NONFINITE = 2    /* some sum was NaN or Inf */
+    GAF_STATUS_NONFINITE = 2,   /* some sum was NaN or Inf */
+    GAF_STATUS_TIMEOUT = 4      /* a bounded wait inside the tensor-core Gram kernel ran out;
+                                   the outputs of that call are not valid */
 };
 
 /* Human-readable name of a return code.  Host only; never NULL. */

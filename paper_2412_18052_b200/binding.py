@@ -14,7 +14,7 @@ import torch
 
 GAF_F32, GAF_BF16 = 0, 1
 GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_GRAM = 0, 1, 2
-GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE = 1, 2
+GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT = 1, 2, 4
 GAF_MAX_K = 64
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgaf.so")

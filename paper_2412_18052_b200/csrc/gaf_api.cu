@@ -7,6 +7,7 @@
 
 #include "../../include/gaf.h"
 #include "gaf_device.cuh"
+#include "gaf_gram_tc.cuh"
 #include "gaf_gramfilter.cuh"
 #include "gaf_pairwise.cuh"
 #include "gaf_stepwise.cuh"
@@ -19,6 +20,7 @@ thread_local int g_launches = 0;
 
 struct DeviceInfo {
     int sms = 0;
+    int l2_bytes = 0;
 };
 
 // Attributes of the current device (queried per call: a cheap driver lookup).
@@ -26,6 +28,7 @@ bool device_info(DeviceInfo *out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&out->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&out->l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return false;
     return out->sms > 0;
 }
 
@@ -70,17 +73,35 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
                                                       2 * gram_matrix_bytes(K));
     a.gram_out = gram_out;
     a.ctl = reinterpret_cast<Control *>(base);
-    // D-slices: fill the machine about twice over all tile pairs, never more than there is work
-    int64_t slices = (int64_t(sms) * 2 + pairs - 1) / pairs;
-    const int64_t work = (D / 4 + kGramThreads - 1) / kGramThreads;
-    if (slices > work) slices = work;
-    if (slices > kGramMaxSlices) slices = kGramMaxSlices;
-    if (slices < 1) slices = 1;
-    a.slices = int(slices);
-    dim3 grid(a.slices, pairs);
-    if (dtype == GAF_F32) gram_tile_kernel<float><<<grid, kGramThreads, 0, st>>>(a);
-    else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
-    ++g_launches;
+    if (dtype == GAF_BF16 && K > kGsMaxK && K <= kTcMaxK) {
+        // tensor cores: one CTA per SM, each with a contiguous slice of D
+        GramTcArgs t{};
+        for (int i = 0; i < K; ++i) t.g[i] = grads[i];
+        t.K = K; t.Kp = K <= 8 ? 8 : (K <= 16 ? 16 : 32); t.D = D;
+        t.partials = a.partials; t.tiles = a.tiles; t.ctl = a.ctl;
+        const int64_t units = D / ((128 / t.Kp) * 64);
+        int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;
+        if (slices > units) slices = units;
+        if (slices < 1) slices = 1;
+        a.slices = int(slices);
+        const int dyn = kTcStages * kTcStageBytes + 1024;
+        if (cudaFuncSetAttribute(gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+            return GAF_ERR_CUDA;
+        gram_tc_kernel<<<a.slices, kTcThreads, dyn, st>>>(t);
+        ++g_launches;
+    } else {
+        // D-slices: fill the machine about twice over all tile pairs, never more than there is work
+        int64_t slices = (int64_t(sms) * 2 + pairs - 1) / pairs;
+        const int64_t work = (D / 4 + kGramThreads - 1) / kGramThreads;
+        if (slices > work) slices = work;
+        if (slices > kGramMaxSlices) slices = kGramMaxSlices;
+        if (slices < 1) slices = 1;
+        a.slices = int(slices);
+        dim3 grid(a.slices, pairs);
+        if (dtype == GAF_F32) gram_tile_kernel<float><<<grid, kGramThreads, 0, st>>>(a);
+        else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
+        ++g_launches;
+    }
     gram_finish_kernel<<<pairs, 256, 0, st>>>(a);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
@@ -121,7 +142,7 @@ int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
 template <typename T>
 int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double tau, const int32_t *ord,
                       float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
-                      unsigned char *base, int sms, cudaStream_t st) {
+                      unsigned char *base, int sms, int l2_bytes, cudaStream_t st) {
     Control *ctl = reinterpret_cast<Control *>(base);
     ReplayArgs r{};
     r.K = K; r.tau = tau; r.mask_out = mask_out; r.dist_out = dist_out; r.count_out = count_out; r.ctl = ctl;
@@ -133,6 +154,10 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
         GramSmallArgs a{};
         for (int t = 0; t < K; ++t) a.g[t] = g[ord[t]];
         a.D = D;
+        // how much of the tail of the Gram pass should stay in L2 for the masked-mean pass
+        const int64_t per_elem = int64_t(K) * int64_t(sizeof(T));
+        const int64_t keep_elems = int64_t(l2_bytes) * 6 / 10 / per_elem;
+        a.keep_from = D > keep_elems ? D - keep_elems : 0;
         a.partials = reinterpret_cast<double *>(base + kExtraOffset);
         a.gram = gram_by_step;
         a.replay = r;
@@ -297,9 +322,9 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
             return rc;
         return dtype == GAF_F32
             ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                       count_out, base, di.sms, st)
+                                       count_out, base, di.sms, di.l2_bytes, st)
             : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                               count_out, base, di.sms, st);
+                                               count_out, base, di.sms, di.l2_bytes, st);
     }
     return dtype == GAF_F32
         ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,

@@ -140,12 +140,17 @@ __device__ __forceinline__ Sums3 block_reduce(Sums3 s, double *scratch) {
 }
 
 // One warp sums `n` per-CTA partial triples in a fixed order (lane-strided, then
-// a shuffle tree).  Every lane must call; lane 0 returns the total.
-__device__ __forceinline__ Sums3 warp_sum_partials(const volatile double *partials, int n) {
+// a shuffle tree).  Every lane must call; lane 0 returns the total.  The partials
+// were published with a fence before the ticket that elected this CTA, so plain
+// L2 loads (which the compiler may issue together) see them.
+__device__ __forceinline__ Sums3 warp_sum_partials(const double *partials, int n) {
     const int lane = threadIdx.x & 31;
     Sums3 s = {0.0, 0.0, 0.0};
+#pragma unroll 4
     for (int i = lane; i < n; i += 32) {
-        s.p += partials[3 * i]; s.na += partials[3 * i + 1]; s.ng += partials[3 * i + 2];
+        const double a = __ldcg(partials + 3 * i), b = __ldcg(partials + 3 * i + 1),
+                     c = __ldcg(partials + 3 * i + 2);
+        s.p += a; s.na += b; s.ng += c;
     }
     return warp_reduce(s);
 }

@@ -1,0 +1,328 @@
+// Tensor-core Gram matrix for bfloat16 micro-gradients (K <= 32): G = X X^T with the
+// D parameters as the contraction axis, on the 5th-generation tensor cores
+// (tcgen05.mma, accumulators in tensor memory).
+//
+// Why tensor cores here: with K = 32 the Gram matrix needs 528 multiply-adds per
+// 64 bytes read, about 107 TFLOP/s at HBM speed -- more than the binary32 pipes
+// deliver, and a fraction of what the tensor pipes do.
+//
+// Shape of one MMA: the K gradients are too few to fill the 128 rows of a tile, so R =
+// 128 / Kp different 64-element chunks of the D axis are stacked in the rows (Kp = K
+// rounded up to 8, 16 or 32): row c*Kp + i holds 64 consecutive elements of gradient i
+// taken from chunk c.  The same shared-memory tile serves as both operands (A = B, both
+// K-major, 128-byte swizzle), so D = A A^T is 128 x 128 and its R diagonal Kp x Kp blocks
+// are R partial Gram matrices; the off-diagonal blocks mix different chunks and are
+// ignored.
+//
+// Pipeline per CTA (one CTA per SM, each with a contiguous slice of D):
+//   warps 4-7  loaders: 16-byte cp.async copies global -> swizzled shared memory, a ring of
+//              kTcStages tiles of 16 KB;
+//   warp 8     one thread issues the MMAs (4 per tile, K = 16 each) into one of two
+//              128-column accumulator buffers in tensor memory and commits to mbarriers;
+//   warps 0-3  epilogue: every kTcDrain tiles read the finished buffer with tcgen05.ld and
+//              add it to binary64 registers (short binary32 accumulation chains only).
+// At the end the R chunk blocks are summed in a fixed order and the CTA writes its partial
+// Gram matrix in the [tile pair][slice][64] layout of the CUDA-core version, so the same
+// finishing kernel totals the slices.  Every wait is bounded.
+#pragma once
+
+#include "gaf_device.cuh"
+
+namespace gaf {
+
+constexpr int kTcThreads = 288;
+constexpr int kTcStages = 6;
+constexpr int kTcStageBytes = 128 * 128;        // 128 rows x 128 bytes
+constexpr int kTcDrain = 8;                     // tiles accumulated in tensor memory between drains
+constexpr int kTcMaxK = 32;
+constexpr int kTcTmemCols = 256;                // two accumulator buffers of 128 columns
+constexpr unsigned int kTcSpinLimit = 1u << 22;
+constexpr int kStatusTimeoutBit = 4;            // GAF_STATUS_TIMEOUT
+
+struct GramTcArgs {
+    const void *g[kTcMaxK];
+    int K;                  // gradients
+    int Kp;                 // 8, 16 or 32
+    int64_t D;
+    double *partials;       // [tile pair][slice][64]
+    int tiles;              // ceil(K / 8)
+    Control *ctl;
+};
+
+// ----------------------------------------------------------------- PTX --------
+
+__device__ __forceinline__ uint32_t tc_smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void tc_mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(tc_smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void tc_mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc_smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool tc_mbar_test(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(tc_smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another thread already gave up.
+__device__ __forceinline__ bool tc_mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    for (unsigned int spin = 0; spin < kTcSpinLimit; ++spin) {
+        if (tc_mbar_test(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (spin > 32) __nanosleep(64);
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tc_cp_async16(uint32_t dst_smem, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+__device__ __forceinline__ void tc_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tc_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void tc_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);       // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                              // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                              // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                              // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, both operands K-major, M = 128, N = 128.
+constexpr uint32_t kTcInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(kTcInstrDesc), "r"(accumulate)
+        : "memory");
+}
+// All MMAs issued so far by this thread arrive on the barrier once they have completed.
+__device__ __forceinline__ void tc_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(bar))
+                 : "memory");
+}
+// 32 lanes x 32 columns of 32-bit accumulators: thread = lane (row), registers = columns.
+__device__ __forceinline__ void tc_tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct GramTcShared {
+    uint64_t full[kTcStages];       // loaders -> MMA: tile landed
+    uint64_t empty[kTcStages];      // MMA -> loaders: tile consumed
+    uint64_t acc_full[2];           // MMA -> epilogue: accumulator buffer complete
+    uint64_t acc_empty[2];          // epilogue -> MMA: accumulator buffer read out
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcArgs a) {
+    extern __shared__ unsigned char tc_dyn_smem[];
+    __shared__ GramTcShared sh;
+
+    // tiles must start on a 1024-byte boundary (swizzle atom)
+    unsigned char *tiles = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(tc_dyn_smem) + 1023) & ~uintptr_t(1023));
+    const uint32_t tiles_u32 = tc_smem_u32(tiles);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int K = a.K, Kp = a.Kp, R = 128 / Kp;
+    const int64_t unit = (int64_t)R * 64;                // elements of D per tile
+    const int64_t n_units = a.D / unit;
+    const int64_t u0 = n_units * blockIdx.x / gridDim.x;
+    const int64_t u1 = n_units * (blockIdx.x + 1) / gridDim.x;
+    const int n_tiles = (int)(u1 - u0);
+    const int n_blocks = (n_tiles + kTcDrain - 1) / kTcDrain;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            tc_mbar_init(&sh.full[s], 128);              // every loader thread arrives
+            tc_mbar_init(&sh.empty[s], 1);               // one commit
+        }
+        for (int b = 0; b < 2; ++b) {
+            tc_mbar_init(&sh.acc_full[b], 1);
+            tc_mbar_init(&sh.acc_empty[b], 128);         // every epilogue thread arrives
+        }
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (blockIdx.x == 0) a.ctl->status = 0;          // first kernel of the operation
+    }
+    // rows of absent gradients (K < Kp) stay zero for the whole kernel
+    if (K < Kp) {
+        for (int idx = threadIdx.x; idx < kTcStages * 128 * 8; idx += kTcThreads) {
+            const int row = (idx >> 3) & 127;
+            if ((row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
+        }
+        tc_fence_async_smem();
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&sh.tmem_base)),
+                     "r"(kTcTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    double gsum[32];                                     // epilogue: this row's 32 loaded columns
+#pragma unroll
+    for (int j = 0; j < 32; ++j) gsum[j] = 0.0;
+
+    if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------ loaders --------
+        const int tl = threadIdx.x - 128;                // 0..127
+        const int pieces = K * R * 8;                    // 16-byte pieces per tile
+        for (int it = 0; it < n_tiles + kTcStages - 1; ++it) {
+            if (it < n_tiles) {
+                const int s = it % kTcStages;
+                bool ok = true;
+                if (it >= kTcStages) ok = tc_mbar_wait(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag);
+                if (!__all_sync(0xFFFFFFFFu, ok)) break;
+                const int64_t e0 = (u0 + it) * unit;     // first element of the tile, per gradient
+                const uint32_t tile = tiles_u32 + (uint32_t)s * kTcStageBytes;
+                for (int p = tl; p < pieces; p += 128) {
+                    const int i = p / (R * 8), rem = p % (R * 8);
+                    const int c = rem >> 3, j = rem & 7;
+                    const int row = c * Kp + i;
+                    const unsigned char *src = static_cast<const unsigned char *>(a.g[i]) +
+                                               (e0 + (int64_t)c * 64 + j * 8) * 2;
+                    tc_cp_async16(tile + row * 128 + ((j ^ (row & 7)) << 4), src);
+                }
+            }
+            tc_cp_async_commit();
+            if (it >= kTcStages - 1) {
+                // this thread's copies of tile it-(kTcStages-1) have landed: make them visible to
+                // the tensor core (asynchronous proxy) and signal
+                tc_cp_async_wait<kTcStages - 1>();
+                tc_fence_async_smem();
+                tc_mbar_arrive(&sh.full[(it - (kTcStages - 1)) % kTcStages]);
+            }
+        }
+        tc_cp_async_wait<0>();
+    } else if (warp == 8) {
+        // ------------------------------------------------------ MMA issuer -----
+        if (lane == 0) {
+            for (int it = 0; it < n_tiles; ++it) {
+                const int s = it % kTcStages;
+                const int blk = it / kTcDrain, buf = blk & 1;
+                const bool first_of_block = (it % kTcDrain) == 0;
+                if (first_of_block && blk >= 2) {
+                    // the epilogue must have read this buffer's previous contents
+                    if (!tc_mbar_wait(&sh.acc_empty[buf], (uint32_t)((blk / 2 - 1) & 1), &sh.abort_flag)) break;
+                }
+                if (!tc_mbar_wait(&sh.full[s], (uint32_t)((it / kTcStages) & 1), &sh.abort_flag)) break;
+                tc_fence_after_sync();
+                const uint64_t desc = tc_smem_desc(tiles_u32 + (uint32_t)s * kTcStageBytes);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    // 16 elements = 32 bytes further along K inside the swizzle atom
+                    const uint64_t dk = desc + (uint64_t)(k * 2);
+                    tc_mma(tmem_base + (uint32_t)buf * 128, dk, dk, (first_of_block && k == 0) ? 0u : 1u);
+                }
+                tc_commit(&sh.empty[s]);
+                if ((it % kTcDrain) == kTcDrain - 1 || it == n_tiles - 1) tc_commit(&sh.acc_full[buf]);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------ epilogue -------
+        for (int blk = 0; blk < n_blocks; ++blk) {
+            const int buf = blk & 1;
+            const bool ok = tc_mbar_wait(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag);
+            if (!__all_sync(0xFFFFFFFFu, ok)) break;      // the load below needs the whole warp
+            tc_fence_after_sync();
+            uint32_t r[32];
+            tc_tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 128 + warp * 32), r);
+            tc_fence_before_sync();
+            tc_mbar_arrive(&sh.acc_empty[buf]);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) gsum[j] += (double)__uint_as_float(r[j]);
+        }
+    }
+
+    // ---------------------------------------------- reduce the R chunk blocks ----
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 8) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols) : "memory");
+    }
+    if (sh.abort_flag) {
+        if (threadIdx.x == 0) atomicOr(&a.ctl->status, kStatusTimeoutBit);
+        return;
+    }
+    // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles <= 32 KB)
+    double *red = reinterpret_cast<double *>(tiles);
+    if (warp < 4) {
+        const int row = warp * 32 + lane;                // row of the 128 x 128 result
+        const int c = row / Kp, i = row % Kp;
+        const int off = c * Kp - warp * 32;              // where this chunk's block starts in the loaded columns
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const int jj = j - off;
+            if (jj >= 0 && jj < Kp) red[((size_t)c * Kp + i) * Kp + jj] = gsum[j];
+        }
+    }
+    __syncthreads();
+    // the elements past the last whole tile (fewer than R * 64 per gradient), first CTA only
+    const int64_t tail0 = n_units * unit;
+    const int tail_len = (int)(a.D - tail0);
+    float *tail = reinterpret_cast<float *>(tiles + 32768);              // [Kp][tail_len] <= 32 KB
+    if (blockIdx.x == 0 && tail_len > 0) {
+        for (int idx = threadIdx.x; idx < K * tail_len; idx += kTcThreads) {
+            const int i = idx / tail_len, e = idx % tail_len;
+            tail[idx] = bf16_bits_to_float(static_cast<const unsigned short *>(a.g[i])[tail0 + e]);
+        }
+    }
+    __syncthreads();
+    const int slices = gridDim.x;
+    for (int e = threadIdx.x; e < Kp * Kp; e += kTcThreads) {
+        const int i = e / Kp, j = e % Kp;
+        if (i > j || j >= K) continue;
+        double s = 0.0;
+        for (int c = 0; c < R; ++c) s += red[((size_t)c * Kp + i) * Kp + j];
+        if (blockIdx.x == 0 && tail_len > 0) {
+            float t = 0.0f;
+            int chain = 0;
+            for (int d = 0; d < tail_len; ++d) {
+                t = fmaf(tail[i * tail_len + d], tail[j * tail_len + d], t);
+                if (++chain == 32) { s += (double)t; t = 0.0f; chain = 0; }
+            }
+            s += (double)t;
+        }
+        const int ti = i >> 3, tj = j >> 3;
+        int tp = 0;
+        for (int r = 0; r < ti; ++r) tp += a.tiles - r;
+        tp += tj - ti;
+        a.partials[((size_t)tp * slices + blockIdx.x) * 64 + (i & 7) * 8 + (j & 7)] = s;
+    }
+}
+
+}  // namespace gaf

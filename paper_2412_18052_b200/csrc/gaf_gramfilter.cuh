@@ -74,23 +74,45 @@ __device__ __forceinline__ void replay_on_gram(const ReplayArgs &r, const volati
 struct GramSmallArgs {
     const void *g[kGsMaxK];                 // processing order
     int64_t D;
+    int64_t keep_from;                      // elements from here on are loaded "keep in L2"
     double *partials;                       // [cta][64]
     double *gram;                           // [K][K]
     ReplayArgs replay;
 };
 
+// 16-byte read-only load with an explicit L2 eviction policy.
+__device__ __forceinline__ uint4 ld16_policy(const void *p, uint64_t policy) {
+    uint4 r;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p), "l"(policy));
+    return r;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
 template <typename T> struct GsVec;         // one 16-byte load per gradient and iteration
 template <> struct GsVec<float> {
     static constexpr int N = 4;
-    static __device__ __forceinline__ void load(const float *base, int64_t e, float (&v)[4]) {
-        float4 a = __ldcs(reinterpret_cast<const float4 *>(base + e));
-        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    static __device__ __forceinline__ void load(const float *base, int64_t e, uint64_t policy, float (&v)[4]) {
+        uint4 r = ld16_policy(base + e, policy);
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y);
+        v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
     }
 };
 template <> struct GsVec<__nv_bfloat16> {
     static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16 *base, int64_t e, float (&v)[8]) {
-        uint4 r = __ldcs(reinterpret_cast<const uint4 *>(base + e));
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *base, int64_t e, uint64_t policy,
+                                                float (&v)[8]) {
+        uint4 r = ld16_policy(base + e, policy);
         unsigned int w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -129,13 +151,18 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
         }
     };
 
+    // The masked-mean pass that follows walks the vectors from their end: the tail of
+    // this pass is loaded "evict last" so that it is still in L2 then; the head, which
+    // cannot survive anyway, is loaded "evict first".
+    const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
     const int64_t n_vec = a.D / N;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int since_flush = 0;
     for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n_vec; q += stride) {
         float x[KT][N];
+        const uint64_t pol = (q * N >= a.keep_from) ? pol_last : pol_first;
 #pragma unroll
-        for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], q * N, x[r]);
+        for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], q * N, pol, x[r]);
         int p = 0;
 #pragma unroll
         for (int r = 0; r < KT; ++r)
@@ -179,10 +206,11 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     __threadfence();
 
     // last CTA: fixed-order totals (one warp per pair), then the scalar walk
-    const volatile double *part = a.partials;
+    const double *part = a.partials;
     for (int p = warp; p < NP; p += kGsThreads / 32) {
         double s = 0.0;
-        for (int i = lane; i < (int)gridDim.x; i += 32) s += part[(size_t)i * 64 + p];
+#pragma unroll 4
+        for (int i = lane; i < (int)gridDim.x; i += 32) s += __ldcg(part + (size_t)i * 64 + p);
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) s += shfl_down_f64(s, d);
         if (lane == 0) {
@@ -223,7 +251,9 @@ struct MaskedMeanArgs {
 };
 
 // out = (((g_0 + g_a) + g_b) + ...) / c over the accepted steps a < b < ..., binary32,
-// in processing order: the same association as the streaming schedules.
+// in processing order: the same association as the streaming schedule.  The vector is
+// walked from its END: the Gram pass that ran just before walked it from the start, so
+// its last-read lines are the ones still in L2.
 template <typename T>
 __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid_constant__ MaskedMeanArgs a) {
     __shared__ const T *list[GAF_MAX_K];
@@ -243,7 +273,7 @@ __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid
     const int64_t n_oct = a.D / kOct;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < n_oct; o += stride) {
-        const int64_t e = o * kOct;
+        const int64_t e = (n_oct - 1 - o) * kOct;
         float v[8];
         load8_stream<T>(list[0], e, v);
         for (int i = 1; i < n; i += 4) {

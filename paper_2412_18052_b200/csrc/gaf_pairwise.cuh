@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(kGramThreads) gram_tile_kernel(GramArgs a) {
         rj[r] = static_cast<const T *>(a.g[j]);
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) a.ctl->status = 0;   // first kernel of the operation
     for (int p = lane; p < kGramTile * kGramTile; p += 32) sacc[warp][p] = 0.0;
     __syncwarp();
 
@@ -142,7 +143,6 @@ __global__ void __launch_bounds__(256) gram_finish_kernel(GramArgs a) {
     int ti, tj;
     tile_pair(blockIdx.x, a.tiles, ti, tj);
     const int p = threadIdx.x & 63, quarter = threadIdx.x >> 6;
-    if (blockIdx.x == 0 && threadIdx.x == 0) a.ctl->status = 0;
     {
         const int per = (a.slices + 3) / 4;
         const int lo = quarter * per, hi = min(a.slices, lo + per);

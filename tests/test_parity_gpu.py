@@ -152,6 +152,14 @@ def test_filter_maximum_k(ws, schedule):
     assert 1 < r["count"] < K
 
 
+@pytest.mark.parametrize("K", [9, 16, 24, 32])
+def test_filter_gram_first_on_tensor_cores(ws, K):
+    """bf16 with 9..32 gradients: the Gram matrix comes from the tcgen05 kernel."""
+    w = _mix(K, 1_000_003 + 64 * K, "bf16", seed=200 + K)
+    r = check_filter(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM)
+    assert 1 < r["count"] < K
+
+
 @pytest.mark.parametrize("schedule", SCHEDULES, ids=SCHED_IDS)
 def test_filter_bitwise_reproducible_and_workspace_reusable(ws, schedule):
     """Fixed-order reductions: two runs agree bit for bit; the workspace needs no
