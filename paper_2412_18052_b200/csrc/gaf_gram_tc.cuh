@@ -14,9 +14,9 @@
 // are R partial Gram matrices; the off-diagonal blocks mix different chunks and are
 // ignored.
 //
-// Pipeline per CTA (one CTA per SM, each with a contiguous slice of D):
+// Pipeline per CTA (one CTA per SM; tiles of the D axis are dealt round-robin to the CTAs):
 //   warps 4-7  loaders: 16-byte cp.async copies global -> swizzled shared memory, a ring of
-//              kTcStages tiles of 16 KB;
+//              kTcStages tiles of 16 KB, each copy batch arriving on the tile's mbarrier by itself;
 //   warp 8     one thread issues the MMAs (4 per tile, K = 16 each) into one of two
 //              128-column accumulator buffers in tensor memory and commits to mbarriers;
 //   warps 0-3  epilogue: every kTcDrain tiles read the finished buffer with tcgen05.ld and
@@ -30,8 +30,17 @@
 
 namespace gaf {
 
-constexpr int kTcThreads = 288;
-constexpr int kTcStages = 6;
+#ifndef GAF_TC_LOADER_WARPS
+#define GAF_TC_LOADER_WARPS 4
+#endif
+#ifndef GAF_TC_STAGES
+#define GAF_TC_STAGES 12
+#endif
+constexpr int kTcLoaderWarps = GAF_TC_LOADER_WARPS;
+constexpr int kTcLoaders = kTcLoaderWarps * 32;
+constexpr int kTcMmaWarp = 4 + kTcLoaderWarps;  // warps 0-3 epilogue, then the loaders, then the MMA issuer
+constexpr int kTcThreads = (kTcMmaWarp + 1) * 32;
+constexpr int kTcStages = GAF_TC_STAGES;
 constexpr int kTcStageBytes = 128 * 128;        // 128 rows x 128 bytes
 constexpr int kTcDrain = 8;                     // tiles accumulated in tensor memory between drains
 constexpr int kTcMaxK = 32;
@@ -76,17 +85,28 @@ __device__ __forceinline__ bool tc_mbar_wait(uint64_t *bar, uint32_t parity, vol
     for (unsigned int spin = 0; spin < kTcSpinLimit; ++spin) {
         if (tc_mbar_test(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (spin > 32) __nanosleep(64);
+        if (spin > 4) __nanosleep(32);
     }
     *abort_flag = 1;
     return false;
 }
+// The same for a whole warp: one lane polls (32 lanes polling one mbarrier are 32 serialised
+// shared-memory operations per round), the others learn the outcome through the shuffle,
+// which also orders their later accesses after the polling lane's acquire.
+__device__ __forceinline__ bool tc_mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = tc_mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
 __device__ __forceinline__ void tc_cp_async16(uint32_t dst_smem, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
 }
-__device__ __forceinline__ void tc_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void tc_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// Asynchronous arrival (counted among the barrier's expected arrivals) once all earlier
+// cp.async copies of this thread have completed.
+__device__ __forceinline__ void tc_cp_async_arrive(uint64_t *bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(tc_smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -154,14 +174,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     const int K = a.K, Kp = a.Kp, R = 128 / Kp;
     const int64_t unit = (int64_t)R * 64;                // elements of D per tile
     const int64_t n_units = a.D / unit;
-    const int64_t u0 = n_units * blockIdx.x / gridDim.x;
-    const int64_t u1 = n_units * (blockIdx.x + 1) / gridDim.x;
-    const int n_tiles = (int)(u1 - u0);
+    // tiles are dealt round-robin to the CTAs, so that at any moment the whole grid reads one
+    // compact window of every gradient (DRAM row locality), not 148 far-apart places
+    const int64_t G = gridDim.x;
+    const int n_tiles = (int)((n_units - blockIdx.x + G - 1) / G);
     const int n_blocks = (n_tiles + kTcDrain - 1) / kTcDrain;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
-            tc_mbar_init(&sh.full[s], 128);              // every loader thread arrives
+            tc_mbar_init(&sh.full[s], kTcLoaders);       // every loader thread arrives
             tc_mbar_init(&sh.empty[s], 1);               // one commit
         }
         for (int b = 0; b < 2; ++b) {
@@ -180,7 +201,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
         }
         tc_fence_async_smem();
     }
-    if (warp == 8) {
+    if (warp == kTcMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&sh.tmem_base)),
                      "r"(kTcTmemCols)
                      : "memory");
@@ -195,38 +216,43 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
 #pragma unroll
     for (int j = 0; j < 32; ++j) gsum[j] = 0.0;
 
-    if (warp >= 4 && warp < 8) {
+    if (warp >= 4 && warp < kTcMmaWarp) {
         // ------------------------------------------------------ loaders --------
-        const int tl = threadIdx.x - 128;                // 0..127
+        const int tl = threadIdx.x - 128;                // 0..kTcLoaders-1
         const int pieces = K * R * 8;                    // 16-byte pieces per tile
-        for (int it = 0; it < n_tiles + kTcStages - 1; ++it) {
-            if (it < n_tiles) {
-                const int s = it % kTcStages;
-                bool ok = true;
-                if (it >= kTcStages) ok = tc_mbar_wait(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag);
-                if (!__all_sync(0xFFFFFFFFu, ok)) break;
-                const int64_t e0 = (u0 + it) * unit;     // first element of the tile, per gradient
-                const uint32_t tile = tiles_u32 + (uint32_t)s * kTcStageBytes;
-                for (int p = tl; p < pieces; p += 128) {
-                    const int i = p / (R * 8), rem = p % (R * 8);
-                    const int c = rem >> 3, j = rem & 7;
-                    const int row = c * Kp + i;
-                    const unsigned char *src = static_cast<const unsigned char *>(a.g[i]) +
-                                               (e0 + (int64_t)c * 64 + j * 8) * 2;
-                    tc_cp_async16(tile + row * 128 + ((j ^ (row & 7)) << 4), src);
-                }
-            }
-            tc_cp_async_commit();
-            if (it >= kTcStages - 1) {
-                // this thread's copies of tile it-(kTcStages-1) have landed: make them visible to
-                // the tensor core (asynchronous proxy) and signal
-                tc_cp_async_wait<kTcStages - 1>();
-                tc_fence_async_smem();
-                tc_mbar_arrive(&sh.full[(it - (kTcStages - 1)) % kTcStages]);
+        // Every tile has the same shape: work out once which pieces this thread copies, from
+        // where (relative to the tile's first element) and to which swizzled position.
+        constexpr int kMaxMine = 128 * 128 / 16 / kTcLoaders;
+        const unsigned char *src_base[kMaxMine];
+        uint32_t dst_off[kMaxMine];
+#pragma unroll
+        for (int k = 0; k < kMaxMine; ++k) {
+            const int p = tl + k * kTcLoaders;
+            src_base[k] = nullptr;
+            dst_off[k] = 0;
+            if (p < pieces) {
+                const int i = p / (R * 8), rem = p % (R * 8);
+                const int c = rem >> 3, j = rem & 7;
+                const int row = c * Kp + i;
+                src_base[k] = static_cast<const unsigned char *>(a.g[i]) + ((int64_t)c * 64 + j * 8) * 2;
+                dst_off[k] = (uint32_t)(row * 128 + ((j ^ (row & 7)) << 4));
             }
         }
-        tc_cp_async_wait<0>();
-    } else if (warp == 8) {
+        for (int it = 0; it < n_tiles; ++it) {
+            const int s = it % kTcStages;
+            if (it >= kTcStages &&
+                !tc_mbar_wait_warp(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag))
+                break;
+            const int64_t byte0 = (blockIdx.x + it * G) * unit * 2;   // first byte of the tile, per gradient
+            const uint32_t tile = tiles_u32 + (uint32_t)s * kTcStageBytes;
+#pragma unroll
+            for (int k = 0; k < kMaxMine; ++k)
+                if (src_base[k] != nullptr) tc_cp_async16(tile + dst_off[k], src_base[k] + byte0);
+            // arrives on the tile's barrier when this thread's copies above have landed
+            tc_cp_async_arrive(&sh.full[s]);
+        }
+        tc_cp_async_wait_all();
+    } else if (warp == kTcMmaWarp) {
         // ------------------------------------------------------ MMA issuer -----
         if (lane == 0) {
             for (int it = 0; it < n_tiles; ++it) {
@@ -255,8 +281,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
         // ------------------------------------------------------ epilogue -------
         for (int blk = 0; blk < n_blocks; ++blk) {
             const int buf = blk & 1;
-            const bool ok = tc_mbar_wait(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag);
-            if (!__all_sync(0xFFFFFFFFu, ok)) break;      // the load below needs the whole warp
+            // (warp-uniform outcome: the load below needs the whole warp)
+            if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag)) break;
             tc_fence_after_sync();
             uint32_t r[32];
             tc_tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 128 + warp * 32), r);
@@ -271,7 +297,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == 8) {
+    if (warp == kTcMmaWarp) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols) : "memory");
     }
     if (sh.abort_flag) {
