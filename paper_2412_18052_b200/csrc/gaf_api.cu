@@ -392,8 +392,22 @@ int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype, 
     DeviceInfo di;
     if (!device_info(&di)) return GAF_ERR_CUDA;
     auto *base = static_cast<unsigned char *>(workspace);
-    return launch_gram_tiles(grads, K, D, dtype, dist_out, gram_out, base, di.sms,
-                             static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (K >= 2 && K <= kGsMaxK) {
+        // few gradients: the one-pass register-tiled Gram kernel, distances in its last CTA
+        GramSmallArgs a{};
+        for (int i = 0; i < K; ++i) a.g[i] = grads[i];
+        a.D = D;
+        a.keep_from = D;                                    // nothing is read again: stream everything
+        a.partials = reinterpret_cast<double *>(base + kExtraOffset);
+        a.gram = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K));
+        a.replay.ctl = reinterpret_cast<Control *>(base);
+        a.pair_dist_out = dist_out;
+        a.pair_gram_out = gram_out;
+        return dtype == GAF_F32 ? launch_gram_small<float>(a, K, di.sms, st)
+                                : launch_gram_small<__nv_bfloat16>(a, K, di.sms, st);
+    }
+    return launch_gram_tiles(grads, K, D, dtype, dist_out, gram_out, base, di.sms, st);
 }
 
 int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out) {

@@ -77,7 +77,9 @@ struct GramSmallArgs {
     int64_t keep_from;                      // elements from here on are loaded "keep in L2"
     double *partials;                       // [cta][64]
     double *gram;                           // [K][K]
-    ReplayArgs replay;
+    ReplayArgs replay;                      // used when pair_dist_out is null
+    float *pair_dist_out;                   // pairwise mode: K x K distances instead of the walk
+    double *pair_gram_out;                  // pairwise mode: optional copy of the Gram matrix
 };
 
 // 16-byte read-only load with an explicit L2 eviction policy.
@@ -129,6 +131,7 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     __shared__ double sacc[kGsThreads / 32][NP];
     __shared__ bool is_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.replay.ctl->status = 0;      // first kernel of the operation
     for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
     __syncwarp();
 
@@ -224,7 +227,21 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     }
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) replay_on_gram(a.replay, a.gram);
+    if (a.pair_dist_out == nullptr) {
+        if (threadIdx.x == 0) replay_on_gram(a.replay, a.gram);
+        return;
+    }
+    // pairwise mode: Eq. 4 for every pair
+    if (threadIdx.x < KT * KT) {
+        const volatile double *G = a.gram;
+        const int i = threadIdx.x / KT, j = threadIdx.x % KT;
+        const double gii = G[i * KT + i], gjj = G[j * KT + j], gij = G[threadIdx.x];
+        int status = 0;
+        const double d = (i == j && gii > 0.0) ? 0.0 : cosine_distance(gij, gii, gjj, &status);
+        a.pair_dist_out[threadIdx.x] = (float)d;
+        if (a.pair_gram_out) a.pair_gram_out[threadIdx.x] = gij;
+        if (status) atomicOr(&a.replay.ctl->status, status);
+    }
 }
 
 // Scalar walk as its own launch (Gram matrix produced by the tiled pairwise kernels).
