@@ -46,6 +46,16 @@ int stream_grid(int64_t D, int threads, int sms) {
     return int(need < cap ? need : cap);
 }
 
+// Which Gram kernel: bfloat16 with up to 32 gradients goes to the tensor cores, except that
+// with at most 8 gradients and a short vector the one-launch register-tiled kernel wins.
+constexpr int64_t kTcMinSmallK = int64_t(1) << 22;
+bool use_tensor_gram(int K, int64_t D, int dtype) {
+    return dtype == GAF_BF16 && K >= 2 && K <= kTcMaxK && (K > kGsMaxK || D >= kTcMinSmallK);
+}
+bool use_small_gram(int K, int64_t D, int dtype) {
+    return K >= 2 && K <= kGsMaxK && !use_tensor_gram(K, D, dtype);
+}
+
 // Layout after the per-CTA triples: Gram partials [tile pair][slice][64] doubles, the
 // Gram matrix by original index, the Gram matrix by processing step, a K x K float
 // scratch for distances nobody asked for.
@@ -73,13 +83,14 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
                                                       2 * gram_matrix_bytes(K));
     a.gram_out = gram_out;
     a.ctl = reinterpret_cast<Control *>(base);
-    if (dtype == GAF_BF16 && K > kGsMaxK && K <= kTcMaxK) {
+    if (use_tensor_gram(K, D, dtype)) {
         // tensor cores: one CTA per SM, each with a contiguous slice of D
         GramTcArgs t{};
         for (int i = 0; i < K; ++i) t.g[i] = grads[i];
         t.K = K; t.Kp = K <= 8 ? 8 : (K <= 16 ? 16 : 32); t.D = D;
         t.partials = a.partials; t.tiles = a.tiles; t.ctl = a.ctl;
-        const int64_t units = D / ((128 / t.Kp) * 64);
+        const int64_t unit = (128 / t.Kp) * 64 * kTcSub;
+        const int64_t units = (D + unit - 1) / unit;
         int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;
         if (slices > units) slices = units;
         if (slices < 1) slices = 1;
@@ -102,7 +113,7 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
         ++g_launches;
     }
-    gram_finish_kernel<<<pairs, 256, 0, st>>>(a);
+    gram_finish_kernel<<<pairs, 64 * kFinishParts, 0, st>>>(a);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }
@@ -150,7 +161,7 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     double *gram_by_index = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K));
     double *gram_by_step = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K) +
                                                       gram_matrix_bytes(K));
-    if (K <= kGsMaxK) {
+    if (use_small_gram(K, D, dtype)) {
         GramSmallArgs a{};
         for (int t = 0; t < K; ++t) a.g[t] = g[ord[t]];
         a.D = D;
@@ -315,7 +326,8 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     if (schedule == GAF_SCHED_AUTO) {
         // Gram-first moves fewer bytes whenever its one-pass Gram kernel applies
         const bool ws_ok = workspace_bytes >= kExtraOffset + pairwise_extra_bytes(K);
-        schedule = (K >= 2 && K <= kGsMaxK && ws_ok) ? GAF_SCHED_GRAM : GAF_SCHED_STEPWISE;
+        const bool fast_gram = K >= 2 && (K <= kGsMaxK || use_tensor_gram(K, D, dtype));
+        schedule = (fast_gram && ws_ok) ? GAF_SCHED_GRAM : GAF_SCHED_STEPWISE;
     }
     if (schedule == GAF_SCHED_GRAM && K >= 2) {
         if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K)))
@@ -393,7 +405,7 @@ int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype, 
     if (!device_info(&di)) return GAF_ERR_CUDA;
     auto *base = static_cast<unsigned char *>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (K >= 2 && K <= kGsMaxK) {
+    if (use_small_gram(K, D, dtype)) {
         // few gradients: the one-pass register-tiled Gram kernel, distances in its last CTA
         GramSmallArgs a{};
         for (int i = 0; i < K; ++i) a.g[i] = grads[i];

@@ -21,6 +21,8 @@
 //              128-column accumulator buffers in tensor memory and commits to mbarriers;
 //   warps 0-3  epilogue: every kTcDrain tiles read the finished buffer with tcgen05.ld and
 //              add it to binary64 registers (short binary32 accumulation chains only).
+// A tile is kTcSub swizzle blocks (kTcSub x 64 elements per row): the issuing thread pays
+// one barrier handshake per tile, which at one block per tile cost more than the MMAs.
 // At the end the R chunk blocks are summed in a fixed order and the CTA writes its partial
 // Gram matrix in the [tile pair][slice][64] layout of the CUDA-core version, so the same
 // finishing kernel totals the slices.  Every wait is bounded.
@@ -31,21 +33,26 @@
 namespace gaf {
 
 #ifndef GAF_TC_LOADER_WARPS
-#define GAF_TC_LOADER_WARPS 4
+#define GAF_TC_LOADER_WARPS 8
 #endif
 #ifndef GAF_TC_STAGES
-#define GAF_TC_STAGES 12
+#define GAF_TC_STAGES 6
+#endif
+#ifndef GAF_TC_SUB
+#define GAF_TC_SUB 2
 #endif
 constexpr int kTcLoaderWarps = GAF_TC_LOADER_WARPS;
 constexpr int kTcLoaders = kTcLoaderWarps * 32;
 constexpr int kTcMmaWarp = 4 + kTcLoaderWarps;  // warps 0-3 epilogue, then the loaders, then the MMA issuer
 constexpr int kTcThreads = (kTcMmaWarp + 1) * 32;
 constexpr int kTcStages = GAF_TC_STAGES;
-constexpr int kTcStageBytes = 128 * 128;        // 128 rows x 128 bytes
-constexpr int kTcDrain = 8;                     // tiles accumulated in tensor memory between drains
+constexpr int kTcSub = GAF_TC_SUB;              // 128-row x 128-byte swizzle blocks per tile (one handshake per tile)
+constexpr int kTcBlockBytes = 128 * 128;        // one such block: 128 rows x 128 bytes
+constexpr int kTcStageBytes = kTcSub * kTcBlockBytes;
+constexpr int kTcDrain = 8 / kTcSub;            // tiles accumulated in tensor memory between drains (32 MMAs)
 constexpr int kTcMaxK = 32;
 constexpr int kTcTmemCols = 256;                // two accumulator buffers of 128 columns
-constexpr unsigned int kTcSpinLimit = 1u << 22;
+constexpr unsigned int kTcSpinLimit = 1u << 19;       // attempts of up to ~2 us each
 constexpr int kStatusTimeoutBit = 4;            // GAF_STATUS_TIMEOUT
 
 struct GramTcArgs {
@@ -69,23 +76,26 @@ __device__ __forceinline__ void tc_mbar_init(uint64_t *bar, uint32_t count) {
 __device__ __forceinline__ void tc_mbar_arrive(uint64_t *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc_smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool tc_mbar_test(uint64_t *bar, uint32_t parity) {
+// One attempt at waiting for the phase with the given parity: the hardware suspends the
+// thread until the phase completes or about `hint_ns` nanoseconds have passed, whichever is
+// first, and wakes it at once on completion (unlike a sleep-and-poll loop, whose sleep
+// granularity would be paid on every tile).
+__device__ __forceinline__ bool tc_mbar_try(uint64_t *bar, uint32_t parity, uint32_t hint_ns) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(tc_smem_u32(bar)), "r"(parity)
+        : "r"(tc_smem_u32(bar)), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
 // Bounded wait: false when the limit ran out or another thread already gave up.
 __device__ __forceinline__ bool tc_mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
     for (unsigned int spin = 0; spin < kTcSpinLimit; ++spin) {
-        if (tc_mbar_test(bar, parity)) return true;
+        if (tc_mbar_try(bar, parity, 2000u)) return true;
         if (*abort_flag) return false;
-        if (spin > 4) __nanosleep(32);
     }
     *abort_flag = 1;
     return false;
@@ -100,6 +110,10 @@ __device__ __forceinline__ bool tc_mbar_wait_warp(uint64_t *bar, uint32_t parity
 }
 __device__ __forceinline__ void tc_cp_async16(uint32_t dst_smem, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+// The same, reading only the first `src_bytes` (0..16) bytes and zero-filling the rest.
+__device__ __forceinline__ void tc_cp_async16_zfill(uint32_t dst_smem, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
 }
 // Asynchronous arrival (counted among the barrier's expected arrivals) once all earlier
 // cp.async copies of this thread have completed.
@@ -172,8 +186,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int K = a.K, Kp = a.Kp, R = 128 / Kp;
-    const int64_t unit = (int64_t)R * 64;                // elements of D per tile
-    const int64_t n_units = a.D / unit;
+    const int64_t unit = (int64_t)R * 64 * kTcSub;       // elements of D per tile and gradient
+    // the last tile may be partial: its missing elements are zero-filled by the copies
+    const int64_t n_units = (a.D + unit - 1) / unit;
     // tiles are dealt round-robin to the CTAs, so that at any moment the whole grid reads one
     // compact window of every gradient (DRAM row locality), not 148 far-apart places
     const int64_t G = gridDim.x;
@@ -195,7 +210,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     }
     // rows of absent gradients (K < Kp) stay zero for the whole kernel
     if (K < Kp) {
-        for (int idx = threadIdx.x; idx < kTcStages * 128 * 8; idx += kTcThreads) {
+        for (int idx = threadIdx.x; idx < kTcStages * kTcSub * 128 * 8; idx += kTcThreads) {
             const int row = (idx >> 3) & 127;
             if ((row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
         }
@@ -219,23 +234,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     if (warp >= 4 && warp < kTcMmaWarp) {
         // ------------------------------------------------------ loaders --------
         const int tl = threadIdx.x - 128;                // 0..kTcLoaders-1
-        const int pieces = K * R * 8;                    // 16-byte pieces per tile
+        const int run = kTcSub * R * 8;                  // 16-byte pieces of one gradient in a tile (contiguous)
+        const int pieces = K * run;                      // 16-byte pieces per tile
         // Every tile has the same shape: work out once which pieces this thread copies, from
         // where (relative to the tile's first element) and to which swizzled position.
-        constexpr int kMaxMine = 128 * 128 / 16 / kTcLoaders;
+        constexpr int kMaxMine = kTcStageBytes / 16 / kTcLoaders;
         const unsigned char *src_base[kMaxMine];
         uint32_t dst_off[kMaxMine];
+        int rel_elem[kMaxMine];                          // element offset of the piece inside the tile
 #pragma unroll
         for (int k = 0; k < kMaxMine; ++k) {
             const int p = tl + k * kTcLoaders;
             src_base[k] = nullptr;
             dst_off[k] = 0;
+            rel_elem[k] = 0;
             if (p < pieces) {
-                const int i = p / (R * 8), rem = p % (R * 8);
-                const int c = rem >> 3, j = rem & 7;
+                const int i = p / run, rem = p % run;
+                const int q = rem >> 3, j = rem & 7;     // 64-element chunk within the run, piece within it
+                const int blk = q / R, c = q % R;        // which swizzle block, which row group
                 const int row = c * Kp + i;
-                src_base[k] = static_cast<const unsigned char *>(a.g[i]) + ((int64_t)c * 64 + j * 8) * 2;
-                dst_off[k] = (uint32_t)(row * 128 + ((j ^ (row & 7)) << 4));
+                rel_elem[k] = q * 64 + j * 8;
+                src_base[k] = static_cast<const unsigned char *>(a.g[i]) + (int64_t)rel_elem[k] * 2;
+                dst_off[k] = (uint32_t)(blk * kTcBlockBytes + row * 128 + ((j ^ (row & 7)) << 4));
             }
         }
         for (int it = 0; it < n_tiles; ++it) {
@@ -243,11 +263,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
             if (it >= kTcStages &&
                 !tc_mbar_wait_warp(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag))
                 break;
-            const int64_t byte0 = (blockIdx.x + it * G) * unit * 2;   // first byte of the tile, per gradient
+            const int64_t elem0 = (blockIdx.x + it * G) * unit;       // first element of the tile, per gradient
+            const int64_t byte0 = elem0 * 2;
             const uint32_t tile = tiles_u32 + (uint32_t)s * kTcStageBytes;
+            if (elem0 + unit <= a.D) {
 #pragma unroll
-            for (int k = 0; k < kMaxMine; ++k)
-                if (src_base[k] != nullptr) tc_cp_async16(tile + dst_off[k], src_base[k] + byte0);
+                for (int k = 0; k < kMaxMine; ++k)
+                    if (src_base[k] != nullptr) tc_cp_async16(tile + dst_off[k], src_base[k] + byte0);
+            } else {
+                // ragged end of the vectors: copy what exists, zero-fill the rest of each piece
+#pragma unroll
+                for (int k = 0; k < kMaxMine; ++k)
+                    if (src_base[k] != nullptr) {
+                        const int64_t left = (a.D - elem0 - rel_elem[k]) * 2;         // bytes that exist from here on
+                        const uint32_t n = left >= 16 ? 16u : (left > 0 ? (uint32_t)left : 0u);
+                        // (a piece that lies wholly past the end reads nothing: point it at the buffer's start)
+                        tc_cp_async16_zfill(tile + dst_off[k], n ? src_base[k] + byte0 : src_base[k] - (int64_t)rel_elem[k] * 2, n);
+                    }
+            }
             // arrives on the tile's barrier when this thread's copies above have landed
             tc_cp_async_arrive(&sh.full[s]);
         }
@@ -265,12 +298,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
                 }
                 if (!tc_mbar_wait(&sh.full[s], (uint32_t)((it / kTcStages) & 1), &sh.abort_flag)) break;
                 tc_fence_after_sync();
-                const uint64_t desc = tc_smem_desc(tiles_u32 + (uint32_t)s * kTcStageBytes);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    // 16 elements = 32 bytes further along K inside the swizzle atom
-                    const uint64_t dk = desc + (uint64_t)(k * 2);
-                    tc_mma(tmem_base + (uint32_t)buf * 128, dk, dk, (first_of_block && k == 0) ? 0u : 1u);
+                for (int b = 0; b < kTcSub; ++b) {
+                    const uint64_t desc = tc_smem_desc(tiles_u32 + (uint32_t)s * kTcStageBytes + b * kTcBlockBytes);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        // 16 elements = 32 bytes further along K inside the swizzle atom
+                        const uint64_t dk = desc + (uint64_t)(k * 2);
+                        tc_mma(tmem_base + (uint32_t)buf * 128, dk, dk, (first_of_block && b == 0 && k == 0) ? 0u : 1u);
+                    }
                 }
                 tc_commit(&sh.empty[s]);
                 if ((it % kTcDrain) == kTcDrain - 1 || it == n_tiles - 1) tc_commit(&sh.acc_full[buf]);
@@ -317,32 +353,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
         }
     }
     __syncthreads();
-    // the elements past the last whole tile (fewer than R * 64 per gradient), first CTA only
-    const int64_t tail0 = n_units * unit;
-    const int tail_len = (int)(a.D - tail0);
-    float *tail = reinterpret_cast<float *>(tiles + 32768);              // [Kp][tail_len] <= 32 KB
-    if (blockIdx.x == 0 && tail_len > 0) {
-        for (int idx = threadIdx.x; idx < K * tail_len; idx += kTcThreads) {
-            const int i = idx / tail_len, e = idx % tail_len;
-            tail[idx] = bf16_bits_to_float(static_cast<const unsigned short *>(a.g[i])[tail0 + e]);
-        }
-    }
-    __syncthreads();
     const int slices = gridDim.x;
     for (int e = threadIdx.x; e < Kp * Kp; e += kTcThreads) {
         const int i = e / Kp, j = e % Kp;
         if (i > j || j >= K) continue;
         double s = 0.0;
         for (int c = 0; c < R; ++c) s += red[((size_t)c * Kp + i) * Kp + j];
-        if (blockIdx.x == 0 && tail_len > 0) {
-            float t = 0.0f;
-            int chain = 0;
-            for (int d = 0; d < tail_len; ++d) {
-                t = fmaf(tail[i * tail_len + d], tail[j * tail_len + d], t);
-                if (++chain == 32) { s += (double)t; t = 0.0f; chain = 0; }
-            }
-            s += (double)t;
-        }
         const int ti = i >> 3, tj = j >> 3;
         int tp = 0;
         for (int r = 0; r < ti; ++r) tp += a.tiles - r;

@@ -137,23 +137,27 @@ __global__ void __launch_bounds__(kGramThreads) gram_tile_kernel(GramArgs a) {
 
 // One CTA per tile pair: sums the slices in a fixed order, writes both triangles of
 // the Gram matrix; the last CTA to finish turns the Gram matrix into distances.
-__global__ void __launch_bounds__(256) gram_finish_kernel(GramArgs a) {
-    __shared__ double part[4][64];
+constexpr int kFinishParts = 16;        // each entry's slices are summed in 16 independent chains
+__global__ void __launch_bounds__(64 * kFinishParts) gram_finish_kernel(GramArgs a) {
+    __shared__ double part[kFinishParts][64];
     __shared__ bool is_last;
     int ti, tj;
     tile_pair(blockIdx.x, a.tiles, ti, tj);
-    const int p = threadIdx.x & 63, quarter = threadIdx.x >> 6;
+    const int p = threadIdx.x & 63, chain = threadIdx.x >> 6;
     {
-        const int per = (a.slices + 3) / 4;
-        const int lo = quarter * per, hi = min(a.slices, lo + per);
+        const int per = (a.slices + kFinishParts - 1) / kFinishParts;
+        const int lo = chain * per, hi = min(a.slices, lo + per);
         double s = 0.0;
         const double *src = a.partials + (size_t)blockIdx.x * a.slices * 64 + p;
-        for (int sl = lo; sl < hi; ++sl) s += src[(size_t)sl * 64];
-        part[quarter][p] = s;
+#pragma unroll 4
+        for (int sl = lo; sl < hi; ++sl) s += __ldcg(src + (size_t)sl * 64);
+        part[chain][p] = s;
     }
     __syncthreads();
     if (threadIdx.x < 64) {
-        double s = (part[0][p] + part[1][p]) + (part[2][p] + part[3][p]);
+        double s = 0.0;
+#pragma unroll
+        for (int c = 0; c < kFinishParts; ++c) s += part[c][p];
         int r = p / kGramTile, c = p % kGramTile;
         int i = ti * kGramTile + r, j = tj * kGramTile + c;
         if (i < a.K && j < a.K && i <= j) {
