@@ -42,8 +42,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=3000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 4, 5],
-                    help="named configuration (2 is the one the metric is quoted on)")
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5],
+                    help="named configuration (2 is the one the metric is quoted on; 3 times the "
+                         "pairwise cosine-distance matrix instead of the filter)")
     ap.add_argument("--tau", type=float, default=0.97)
     ap.add_argument("--schedule", type=int, default=0, help="0 auto, 1 stepwise (streaming), 2 Gram-first")
     ap.add_argument("--e2e-steps", type=int, default=10)
@@ -75,6 +76,35 @@ def gram_first_bytes(mask_in_order, K, D, b):
         return (b + 4) * D
     c = sum(int(x) for x in mask_in_order)
     return ((K + c) * b + 4) * D
+
+
+# DRAM traffic (dram__bytes_read + dram__bytes_write) of the kernels of one call, from the ncu
+# capture summarised in profiles/gram_first_config2.md.  Reported only while the kernel sources
+# are the ones that were profiled (their hash is checked); otherwise `traffic` is null.
+NCU_TRAFFIC = {
+    "sources": ["paper_2412_18052_b200/csrc/gaf_gramfilter.cuh", "paper_2412_18052_b200/csrc/gaf_device.cuh"],
+    "sha256": "TO-BE-RECORDED",
+    "gram_small_kernel<float,4>": 183.35e6,                 # per launch, configuration 2
+    "masked_mean_kernel<float>": {3: 151.89e6, 2: 102.33e6},  # per launch, by accepted count c
+}
+
+
+def ncu_traffic_config2(masks, n_sets, steps):
+    """Average DRAM bytes per call over the rotating input sets, or None."""
+    import hashlib
+    h = hashlib.sha256()
+    for rel in NCU_TRAFFIC["sources"]:
+        with open(os.path.join(ROOT, rel), "rb") as fh:
+            h.update(fh.read())
+    if h.hexdigest() != NCU_TRAFFIC["sha256"]:
+        return None
+    per_set = []
+    for m in masks:
+        c = sum(int(x) for x in m)
+        if c not in NCU_TRAFFIC["masked_mean_kernel<float>"]:
+            return None
+        per_set.append(NCU_TRAFFIC["gram_small_kernel<float,4>"] + NCU_TRAFFIC["masked_mean_kernel<float>"][c])
+    return sum(per_set[i % n_sets] for i in range(steps)) / steps
 
 
 # ---------------------------------------------------------------- clocks -----
@@ -142,6 +172,8 @@ def time_oracle(cfg: int, tau: float, seconds: float):
     from oracle import gaf_oracle as orc
     from paper_2412_18052_b200 import workloads
 
+    if cfg == 3:
+        cfg = 2                     # the reference arm times the filter; 3 is the pairwise matrix
     full = {1: 1_000_000, 2: workloads.RESNET18_100_NUMEL, 4: workloads.GPT2_SMALL_NUMEL,
             5: 1_000_000_000}[cfg]
     # configurations 4 and 5 are sampled at reduced D (same recipe) to bound the run
@@ -187,6 +219,62 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------ ours -----
+
+def run_pairwise(args):
+    """Configuration 3: the K x K pairwise cosine-distance matrix (one GPU)."""
+    import torch
+
+    import paper_2412_18052_b200 as gaf
+    from paper_2412_18052_b200 import workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(0)
+    w = workloads.config(3, device="cuda:0")
+    K, D, b = w.K, w.D, w.elem_bytes
+    ws = gaf.new_workspace(K, D, gaf.GAF_BF16, device="cuda:0")
+    dist_out = torch.empty(K, K, dtype=torch.float32, device="cuda:0")
+    gram = torch.empty(K, K, dtype=torch.float64, device="cuda:0")
+
+    def step():
+        gaf.gaf_pairwise_cosdist(w.grads, ws, dist_out=dist_out, gram_out=gram)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    launches = gaf.gaf_last_launch_count()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    in_bytes = K * b * D
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_kind = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_kind = 6650.0, "fallback"
+    achieved = in_bytes / (ms * 1e-3) / 1e9
+    line = {
+        "metric": "gaf_pairwise_cosdist micro-gradient GB/s", "value": achieved, "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32 (tensor cores), f64 sums",
+        "data": "synthetic",
+        "config": {"workload": f"configuration 3: pairwise matrix, K={K}, D={D}, bf16 inputs", "K": K, "D": D,
+                   "l2": f"inputs of one call ({in_bytes / 1e6:.0f} MB) exceed the 126 MB L2"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "kernel": "gram_tc_kernel + gram_finish_kernel (whole call)",
+                     "byte_model": "every gradient read once: K b D", "algorithmic_bytes_per_launch": in_bytes},
+        "e2e": None, "gpu_launches": launches * args.steps, "clocks": clocks, "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+
 
 def run_ours(args):
     import torch
@@ -337,7 +425,9 @@ def run_ours(args):
             },
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak,
+                "traffic": (ncu_traffic_config2(masks, n_sets, n_launch_timed)
+                            if (cfg == 2 and sched_used == 2 and abs(args.tau - 0.97) < 1e-12) else None),
                 "peak_kind": f"of {peak_kind}",
                 "kernel": ("gram_small_kernel + masked_mean_kernel (whole call, both HBM-streaming)"
                            if sched_used == 2 else "step_kernel x%d (whole call)" % launches_per_step),
@@ -361,6 +451,9 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == 3:
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_pairwise(args)
     else:
         run_ours(args)
 
