@@ -83,7 +83,7 @@ def gram_first_bytes(mask_in_order, K, D, b):
 # are the ones that were profiled (their hash is checked); otherwise `traffic` is null.
 NCU_TRAFFIC = {
     "sources": ["paper_2412_18052_b200/csrc/gaf_gramfilter.cuh", "paper_2412_18052_b200/csrc/gaf_device.cuh"],
-    "sha256": "TO-BE-RECORDED",
+    "sha256": "b5091e5225a1a605cccb05d943c19fb8f18c1677363bcca64bb366a1785c80b8",
     "gram_small_kernel<float,4>": 183.35e6,                 # per launch, configuration 2
     "masked_mean_kernel<float>": {3: 151.89e6, 2: 102.33e6},  # per launch, by accepted count c
 }
@@ -218,6 +218,25 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------- replicas over ranks --
+
+def max_over_ranks(value: float, device: str = "cpu") -> float:
+    """The slowest rank sets the time of a multi-replica run (MAX all-reduce; works with the
+    gloo backend on CPU tensors and with nccl on CUDA tensors)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gbs(world: int, bytes_per_replica_step: float, ms_per_step: float) -> float:
+    """Whole-job rate of `world` independent replicas that all took `ms_per_step`."""
+    return world * bytes_per_replica_step / (ms_per_step * 1e-3) / 1e9
+
+
 # ------------------------------------------------------------------ ours -----
 
 def run_pairwise(args):
@@ -342,14 +361,10 @@ def run_ours(args):
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.stop()
-    elapsed_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(ev0.elapsed_time(ev1), dev)
     ms_per_step = elapsed_ms / steps
     grad_bytes = K * b * D
-    value = world * grad_bytes / (ms_per_step * 1e-3) / 1e9
+    value = aggregate_gbs(world, grad_bytes, ms_per_step)
 
     # dominant kernel, timed per launch with events on the launching stream
     n_launch_timed = min(steps, 200)
@@ -392,12 +407,8 @@ def run_ours(args):
         for i in range(n_e2e):
             e2e_step(i)                       # synchronises the stream itself
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * grad_bytes / (dt / n_e2e) / 1e9, "unit": UNIT,
+        dt = max_over_ranks(time.perf_counter() - t0, dev)
+        e2e = {"value": aggregate_gbs(world, grad_bytes, dt / n_e2e * 1e3), "unit": UNIT,
                "h2d_bytes_per_step": grad_bytes, "d2h_bytes_per_step": 4 * D + K + 4 * K + 4,
                "steps": n_e2e}
 
