@@ -145,6 +145,42 @@ int gaf_oracle_filter_accumulate(const void *const *grads, int K, int64_t D,
 }
 
 /*
+ * Order-indifferent variant sketched at the end of Section 3.1: every micro-gradient
+ * in turn acts as the initial one and the others follow "around the ring", i.e. for
+ * seed s the processing order is s, s+1, ..., K-1, 0, ..., s-1; Algorithm 1 runs on
+ * each of the K orders and the result with the largest agreement is kept.
+ * Reading taken where the paper leaves it open: agreement = the accepted count c;
+ * ties go to the smallest s.                                 [parity unpinned]
+ *   g, mask, dist, count   as in gaf_oracle_filter_accumulate, for the winning seed
+ *   seed_out               the winning seed
+ *   counts_out             NULL or K entries: c obtained with each seed
+ *   work                   D doubles of scratch
+ */
+int gaf_oracle_filter_any_seed(const void *const *grads, int K, int64_t D, int dtype,
+                               double tau, double *g, uint8_t *mask, double *dist,
+                               int32_t *count, int32_t *seed_out, int32_t *counts_out,
+                               double *work)
+{
+    if (K < 1 || K > 4096) return 1;
+    int32_t order[4096];
+    uint8_t m[4096];
+    double dd[4096];
+    int best_seed = -1;
+    int32_t best_count = 0;
+    for (int s = 0; s < K; ++s) {
+        for (int t = 0; t < K; ++t) order[t] = (s + t) % K;
+        int32_t c = 0;
+        gaf_oracle_filter_accumulate(grads, K, D, dtype, tau, order, NULL, work, m, dd, &c, NULL);
+        if (counts_out) counts_out[s] = c;
+        if (c > best_count) { best_count = c; best_seed = s; }
+    }
+    for (int t = 0; t < K; ++t) order[t] = (best_seed + t) % K;
+    gaf_oracle_filter_accumulate(grads, K, D, dtype, tau, order, NULL, g, mask, dist, count, NULL);
+    *seed_out = best_seed;
+    return 0;
+}
+
+/*
  * Pairwise cosine distances between K micro-gradients (the quantity the
  * paper's cosine-distance figures plot).  gram and dist are K*K row-major.
  * Diagonal: 0 when the norm is non-zero; rows/columns of a zero-norm vector

@@ -64,6 +64,8 @@ def _load():
         vp, i64, i32, dbl = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_double
         lib.gaf_oracle_cosdist.argtypes = [vp, vp, i64, i32, vp, vp]
         lib.gaf_oracle_filter_accumulate.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, vp]
+        lib.gaf_oracle_filter_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, vp]
+        lib.gaf_oracle_filter_any_seed.restype = ctypes.c_int
         lib.gaf_oracle_pairwise.argtypes = [vp, i32, i64, i32, vp, vp]
         lib.gaf_oracle_plain_average.argtypes = [vp, i32, i64, i32, vp]
         for f in (lib.gaf_oracle_cosdist, lib.gaf_oracle_filter_accumulate,
@@ -150,6 +152,28 @@ def filter_accumulate(grads: Sequence[np.ndarray], tau: float,
     if rc != 0:
         raise ValueError("oracle rejected its arguments")
     return FilterResult(out, mask, dist, int(count.value), stats)
+
+
+def filter_any_seed(grads: Sequence[np.ndarray], tau: float):
+    """Order-indifferent variant (end of Section 3.1): Algorithm 1 from every seed in ring
+    order, keep the largest accepted count (ties: smallest seed).
+    Returns (FilterResult of the winner, seed, counts per seed)."""
+    arrs, ptrs, code, D = _prep(grads)
+    K = len(arrs)
+    out = np.empty(D, dtype=np.float64)
+    work = np.empty(D, dtype=np.float64)
+    mask = np.zeros(K, dtype=np.uint8)
+    dist = np.zeros(K, dtype=np.float64)
+    counts = np.zeros(K, dtype=np.int32)
+    count, seed = ctypes.c_int32(), ctypes.c_int32()
+    rc = _load().gaf_oracle_filter_any_seed(
+        ctypes.cast(ptrs, ctypes.c_void_p), K, D, code, float(tau), out.ctypes.data,
+        mask.ctypes.data, dist.ctypes.data, ctypes.addressof(count), ctypes.addressof(seed),
+        counts.ctypes.data, work.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle rejected its arguments")
+    res = FilterResult(out, mask, dist, int(count.value), np.zeros((K, 3)))
+    return res, int(seed.value), counts
 
 
 def pairwise_cosdist(grads: Sequence[np.ndarray]):

@@ -368,6 +368,34 @@ def pin_closed_form_mixture():
     assert [round(float(x), 2) for x in r.dist] == [0.0, 0.33, 1.0, 1.5]
 
 
+def pin_any_seed_variant():
+    """Order-indifferent variant: it is Algorithm 1 run from every seed in ring order with
+    the largest count kept (checked against the plain routine, seed by seed), and it rescues
+    Section 3.1's degenerate example of a first gradient orthogonal to all others."""
+    e = f32(0, 0, 0, 1)
+    a = f32(1, 0.1, 0, 0)
+    b = f32(1, -0.1, 0.1, 0)
+    c = f32(0.9, 0, -0.1, 0)
+    gs = [e, a, b, c]
+    plain = orc.filter_accumulate(gs, 0.5)
+    assert plain.count == 1                                  # the whole macrobatch would be wasted
+    r, seed, counts = orc.filter_any_seed(gs, 0.5)
+    assert seed == 1 and r.count == 3 and r.mask.tolist() == [0, 1, 1, 1]
+    assert counts.tolist() == [1, 3, 3, 3]                   # ties go to the smallest seed
+    assert np.allclose(r.out, (a.astype(np.float64) + b + c) / 3, rtol=1e-15)
+    rng = np.random.RandomState(12)
+    for K, D, tau in ((3, 7, 0.6), (5, 40, 0.8), (6, 129, 0.97)):
+        gs = _rand_grads(rng, K, D, "f32", shared=0.4)
+        gs[1] = (-gs[0]).astype(np.float32)
+        r, seed, counts = orc.filter_any_seed(gs, tau)
+        per_seed = [orc.filter_accumulate(gs, tau, order=[(s + t) % K for t in range(K)]) for s in range(K)]
+        assert counts.tolist() == [p.count for p in per_seed]
+        best = max(range(K), key=lambda s: (per_seed[s].count, -s))
+        assert seed == best and r.count == per_seed[best].count
+        assert r.mask.tolist() == per_seed[best].mask.tolist()
+        assert np.array_equal(r.out, per_seed[best].out) and np.array_equal(r.dist, per_seed[best].dist)
+
+
 ALL_PINS = [
     pin_stated_values,
     pin_figure2_angles,
@@ -384,4 +412,5 @@ ALL_PINS = [
     pin_bilinearity_ties_filter_to_pairwise,
     pin_forced_decisions,
     pin_closed_form_mixture,
+    pin_any_seed_variant,
 ]

@@ -39,6 +39,12 @@ MUTANTS = [
     ("pairwise_wrong_norm", "gram[i * K + i], gram[j * K + j]);", "gram[i * K + i], gram[i * K + i]);"),
     ("forced_ignored", "if (forced && forced[t] >= 0) accept = forced[t];", ""),
     ("average_not_divided", "out[d] = sum / (double)K;", "out[d] = sum;"),
+    ("ring_order_not_rotated", "for (int t = 0; t < K; ++t) order[t] = (s + t) % K;",
+     "for (int t = 0; t < K; ++t) order[t] = t;"),
+    ("ring_ties_to_last", "if (c > best_count) { best_count = c; best_seed = s; }",
+     "if (c >= best_count) { best_count = c; best_seed = s; }"),
+    ("ring_keeps_smallest", "if (c > best_count) { best_count = c; best_seed = s; }",
+     "if (best_seed < 0 || c < best_count) { best_count = c; best_seed = s; }"),
 ]
 
 
