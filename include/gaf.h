@@ -150,6 +150,27 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
                           int schedule, void *cuda_stream);
 
 /*
+ * Order-indifferent variant, as sketched at the end of Section 3.1: Algorithm 1 is
+ * order dependent (a first gradient orthogonal to all others wastes the whole
+ * macrobatch), so every micro-gradient in turn acts as the initial one, the
+ * others following in ring order s, s+1, ..., K-1, 0, ..., s-1, and the result
+ * with the largest agreement is kept.  Where the paper leaves it open: agreement
+ * is the accepted count c; ties go to the smallest s.  All K walks run on one
+ * K x K Gram matrix (dot products are bilinear), so the cost is that of
+ * gaf_filter_accumulate with GAF_SCHED_GRAM: every gradient read once, the
+ * accepted ones once more.
+ *   mask_out, dist_out, count_out, macro_out   as in gaf_filter_accumulate, for
+ *               the winning seed (dist[seed] = 0); the accepted gradients are added
+ *               in the winning ring order
+ *   seed_out    device, 1 int32: the winning seed
+ */
+int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, int dtype,
+                                   double tau,
+                                   float *macro_out, uint8_t *mask_out, float *dist_out,
+                                   int32_t *count_out, int32_t *seed_out,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The same operation for gradients that live in HOST memory (pinned memory
  * makes the copies asynchronous and fast).  Copies each gradient to the device
  * staging area, runs gaf_filter_accumulate, copies the results back and

@@ -24,6 +24,7 @@ EXPORTS = [
     "gaf_error_string", "gaf_workspace_bytes", "gaf_workspace_init", "gaf_cosdist",
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
     "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
+    "gaf_filter_accumulate_any_seed",
 ]
 
 
@@ -57,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.gaf_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.gaf_last_launch_count.argtypes = []
         L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+        L.gaf_filter_accumulate_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS:
             if name != "gaf_error_string":
                 getattr(L, name).restype = i32
@@ -173,6 +175,27 @@ def gaf_filter_accumulate(grads: Sequence[torch.Tensor], tau: float, workspace: 
                                        count_out.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                        int(schedule), _stream()), "gaf_filter_accumulate")
     return macro_out, mask_out, dist_out, count_out
+
+
+def gaf_filter_accumulate_any_seed(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,
+                                   macro_out: Optional[torch.Tensor] = None):
+    """Order-indifferent variant (end of Section 3.1): every gradient in turn is the seed, ring
+    order, largest accepted count wins.  Returns (macro, mask, dist, count, seed) device tensors."""
+    K, D = len(grads), grads[0].numel()
+    dev = grads[0].device
+    if macro_out is None:
+        macro_out = torch.empty(D, dtype=torch.float32, device=dev)
+    mask_out = torch.empty(K, dtype=torch.uint8, device=dev)
+    dist_out = torch.empty(K, dtype=torch.float32, device=dev)
+    count_out = torch.empty(1, dtype=torch.int32, device=dev)
+    seed_out = torch.empty(1, dtype=torch.int32, device=dev)
+    ptrs = _ptr_array(grads)
+    _check(lib().gaf_filter_accumulate_any_seed(
+        ctypes.cast(ptrs, ctypes.c_void_p), K, D, _dtype_code(grads[0]), float(tau),
+        macro_out.data_ptr(), mask_out.data_ptr(), dist_out.data_ptr(), count_out.data_ptr(),
+        seed_out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
+        "gaf_filter_accumulate_any_seed")
+    return macro_out, mask_out, dist_out, count_out, seed_out
 
 
 def gaf_filter_accumulate_host(grads_host: Sequence[torch.Tensor], tau: float,

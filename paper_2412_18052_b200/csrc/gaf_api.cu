@@ -150,11 +150,17 @@ int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
 }
 
 // Gram-first schedule: Gram matrix, scalar walk of Algorithm 1, masked mean.
+// `seed_out` non-null selects the any-seed variant (ord must then be the identity).
 template <typename T>
 int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double tau, const int32_t *ord,
                       float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
-                      unsigned char *base, int sms, int l2_bytes, cudaStream_t st) {
+                      int32_t *seed_out, unsigned char *base, int sms, int l2_bytes, cudaStream_t st) {
     Control *ctl = reinterpret_cast<Control *>(base);
+    RingArgs ring{};
+    if (seed_out) {
+        ring.K = K; ring.tau = tau; ring.mask_out = mask_out; ring.dist_out = dist_out;
+        ring.count_out = count_out; ring.seed_out = seed_out; ring.ctl = ctl;
+    }
     ReplayArgs r{};
     r.K = K; r.tau = tau; r.mask_out = mask_out; r.dist_out = dist_out; r.count_out = count_out; r.ctl = ctl;
     for (int t = 0; t < K; ++t) r.idx[t] = ord[t];
@@ -172,10 +178,12 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
         a.partials = reinterpret_cast<double *>(base + kExtraOffset);
         a.gram = gram_by_step;
         a.replay = r;
+        a.ring = ring;
         if (int rc = launch_gram_small<T>(a, K, sms, st)) return rc;
     } else {
         if (int rc = launch_gram_tiles(g, K, D, dtype, nullptr, nullptr, base, sms, st)) return rc;
-        gram_replay_kernel<<<1, 256, 0, st>>>(r, gram_by_index, gram_by_step);
+        if (seed_out) gram_ring_replay_kernel<<<1, GAF_MAX_K, 0, st>>>(ring, gram_by_index);
+        else gram_replay_kernel<<<1, 256, 0, st>>>(r, gram_by_index, gram_by_step);
         ++g_launches;
     }
     MaskedMeanArgs m{};
@@ -334,15 +342,58 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
             return rc;
         return dtype == GAF_F32
             ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                       count_out, base, di.sms, di.l2_bytes, st)
+                                       count_out, nullptr, base, di.sms, di.l2_bytes, st)
             : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                               count_out, base, di.sms, di.l2_bytes, st);
+                                               count_out, nullptr, base, di.sms, di.l2_bytes, st);
     }
     return dtype == GAF_F32
         ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
                                  ctl, partials, di.sms, st)
         : launch_stepwise<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
                                          count_out, ctl, partials, di.sms, st);
+}
+
+int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, int dtype, double tau,
+                                   float *macro_out, uint8_t *mask_out, float *dist_out,
+                                   int32_t *count_out, int32_t *seed_out, void *workspace,
+                                   size_t workspace_bytes, void *cuda_stream) {
+    g_launches = 0;
+    if (int rc = check_grads(grads, K, D, dtype)) return rc;
+    if ((!macro_out && D > 0) || !mask_out || !count_out || !seed_out) return GAF_ERR_ARG;
+    if (tau != tau) return GAF_ERR_ARG;
+    if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
+    {
+        const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
+        for (int i = 0; i < K; ++i) {
+            const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
+            const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
+            if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
+        }
+    }
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K))) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t ord[GAF_MAX_K];
+    for (int t = 0; t < K; ++t) ord[t] = t;
+    if (K == 1) {
+        // one gradient: it is the seed and the result
+        Control *ctl = reinterpret_cast<Control *>(base);
+        double *partials = reinterpret_cast<double *>(base + kPartialsOffset);
+        int rc = dtype == GAF_F32
+            ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out, ctl,
+                                     partials, di.sms, st)
+            : launch_stepwise<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
+                                             ctl, partials, di.sms, st);
+        if (rc != GAF_OK) return rc;
+        return cudaMemsetAsync(seed_out, 0, sizeof(int32_t), st) == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+    }
+    return dtype == GAF_F32
+        ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out, count_out,
+                                   seed_out, base, di.sms, di.l2_bytes, st)
+        : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
+                                           count_out, seed_out, base, di.sms, di.l2_bytes, st);
 }
 
 int gaf_host_staging_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {

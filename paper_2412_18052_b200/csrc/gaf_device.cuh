@@ -21,7 +21,7 @@ struct Control {
     unsigned int reserved1;
     int status;                         // GAF_STATUS_* bits of the latest call
     int count;                          // running c of Algorithm 1
-    int pad;
+    int ring_seed;                      // any-seed variant: the winning seed, else -1
     unsigned long long accept_bits;     // Gram-first schedule: bit t set = step t accepted
     int decision[GAF_MAX_K];            // by step t: 1 accept, 0 reject
     double sums[GAF_MAX_K][3];          // by step t: {g_i.g, |g|^2, |g_i|^2}

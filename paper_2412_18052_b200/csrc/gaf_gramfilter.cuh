@@ -63,10 +63,84 @@ __device__ __forceinline__ void replay_on_gram(const ReplayArgs &r, const volati
         }
     }
     c->accept_bits = bits;
+    c->ring_seed = -1;
     c->count = count;
     c->status = status;
     *r.count_out = count;
     __threadfence();
+}
+
+// Order-indifferent variant (end of Section 3.1): Algorithm 1 from every seed s with the
+// others following in ring order s, s+1, ..., K-1, 0, ..., s-1; the seed with the largest
+// accepted count wins, ties to the smallest s.  Threads 0..K-1 of the calling block each walk
+// one seed on the Gram matrix (by ORIGINAL index); thread 0 then publishes the winner.
+// `scratch` holds K ints + K unsigned long longs in shared memory.  All threads must call.
+struct RingArgs {
+    int K;
+    double tau;
+    uint8_t *mask_out;
+    float *dist_out;                        // may be null
+    int32_t *count_out;
+    int32_t *seed_out;
+    Control *ctl;
+};
+
+__device__ __forceinline__ void ring_walk_one_seed(const RingArgs &r, const volatile double *gram, int s,
+                                                   int &count_out, unsigned long long &bits_out, int &status_out,
+                                                   float *dist_by_index) {
+    const int K = r.K;
+    unsigned long long bits = 1ull << s;    // bit i set = gradient i (original index) accepted
+    int count = 1, status = 0;
+    double na = gram[(size_t)s * K + s];
+    if (dist_by_index) dist_by_index[s] = 0.0f;
+    for (int t = 1; t < K; ++t) {
+        const int i = (s + t) % K;
+        double p = 0.0;
+        for (int u = 0; u < t; ++u) {       // accepted gradients in processing order
+            const int j = (s + u) % K;
+            if ((bits >> j) & 1ull) p += gram[(size_t)j * K + i];
+        }
+        const double ng = gram[(size_t)i * K + i];
+        const double d = cosine_distance(p, na, ng, &status);
+        if (dist_by_index) dist_by_index[i] = (float)d;
+        if (d <= r.tau) {
+            bits |= 1ull << i;
+            na = na + 2.0 * p + ng;
+            ++count;
+        }
+    }
+    count_out = count; bits_out = bits; status_out = status;
+}
+
+__device__ __forceinline__ void ring_replay_on_gram(const RingArgs &r, const volatile double *gram,
+                                                    int *sh_count, unsigned long long *sh_bits) {
+    const int K = r.K;
+    if ((int)threadIdx.x < K) {
+        int c, st;
+        unsigned long long b;
+        ring_walk_one_seed(r, gram, threadIdx.x, c, b, st, nullptr);
+        sh_count[threadIdx.x] = c;
+        sh_bits[threadIdx.x] = b;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int best = 0;
+        for (int s = 1; s < K; ++s)
+            if (sh_count[s] > sh_count[best]) best = s;
+        // walk the winner once more to write its distances and status
+        int c, st;
+        unsigned long long b;
+        ring_walk_one_seed(r, gram, best, c, b, st, r.dist_out);
+        for (int i = 0; i < K; ++i) r.mask_out[i] = (uint8_t)((b >> i) & 1ull);
+        Control *ctl = r.ctl;
+        ctl->accept_bits = b;
+        ctl->ring_seed = best;
+        ctl->count = c;
+        ctl->status = st;
+        *r.count_out = c;
+        *r.seed_out = best;
+        __threadfence();
+    }
 }
 
 // ------------------------------------------------ one-pass Gram for K <= 8 ----
@@ -77,9 +151,10 @@ struct GramSmallArgs {
     int64_t keep_from;                      // elements from here on are loaded "keep in L2"
     double *partials;                       // [cta][64]
     double *gram;                           // [K][K]
-    ReplayArgs replay;                      // used when pair_dist_out is null
+    ReplayArgs replay;                      // used when pair_dist_out is null and ring.K == 0
     float *pair_dist_out;                   // pairwise mode: K x K distances instead of the walk
     double *pair_gram_out;                  // pairwise mode: optional copy of the Gram matrix
+    RingArgs ring;                          // any-seed mode when ring.K > 0 (rows are in original order)
 };
 
 // 16-byte read-only load with an explicit L2 eviction policy.
@@ -227,6 +302,12 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     }
     __threadfence();
     __syncthreads();
+    if (a.ring.K > 0) {
+        __shared__ int ring_count[kGsMaxK];
+        __shared__ unsigned long long ring_bits[kGsMaxK];
+        ring_replay_on_gram(a.ring, a.gram, ring_count, ring_bits);
+        return;
+    }
     if (a.pair_dist_out == nullptr) {
         if (threadIdx.x == 0) replay_on_gram(a.replay, a.gram);
         return;
@@ -257,10 +338,19 @@ __global__ void gram_replay_kernel(ReplayArgs r, const double *gram_by_index, do
     if (threadIdx.x == 0) replay_on_gram(r, gram_by_step);
 }
 
+// Any-seed walk as its own launch (Gram matrix by original index from the tiled or
+// tensor-core kernels).  One block of at least K threads.
+__global__ void gram_ring_replay_kernel(RingArgs r, const double *gram_by_index) {
+    __shared__ int ring_count[GAF_MAX_K];
+    __shared__ unsigned long long ring_bits[GAF_MAX_K];
+    ring_replay_on_gram(r, gram_by_index, ring_count, ring_bits);
+}
+
 // ------------------------------------------------------- masked mean (Eq. 5) --
 
 struct MaskedMeanArgs {
-    const void *g[GAF_MAX_K];               // processing order
+    const void *g[GAF_MAX_K];               // processing order; original order in any-seed mode, where
+                                            // the order starts at the winning seed and wraps around
     int K;
     int64_t D;
     float *out;
@@ -278,9 +368,13 @@ __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid
     __shared__ float cdiv_s;
     if (threadIdx.x == 0) {
         const unsigned long long bits = *reinterpret_cast<const volatile unsigned long long *>(&a.ctl->accept_bits);
+        const int seed = *reinterpret_cast<const volatile int *>(&a.ctl->ring_seed);
+        const int start = seed < 0 ? 0 : seed;
         int n = 0;
-        for (int t = 0; t < a.K; ++t)
-            if ((bits >> t) & 1ull) list[n++] = static_cast<const T *>(a.g[t]);
+        for (int t = 0; t < a.K; ++t) {
+            const int i = (start + t) % a.K;
+            if ((bits >> i) & 1ull) list[n++] = static_cast<const T *>(a.g[i]);
+        }
         n_list = n;
         cdiv_s = (float)n;
     }

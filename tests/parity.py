@@ -133,3 +133,27 @@ def check_pairwise(grads: Sequence[torch.Tensor], workspace: torch.Tensor):
     for i in range(K):
         assert g_dist[i, i] == (0.0 if o_gram[i, i] > 0 else 1.0)
     return err
+
+
+def check_any_seed(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor):
+    """gaf_filter_accumulate_any_seed against the oracle: the winning seed, and for that
+    seed everything check_filter checks (ring order starting at the seed)."""
+    K = len(grads)
+    macro, mask, dist, count, seed = gaf.gaf_filter_accumulate_any_seed(grads, tau, workspace)
+    np_grads = [as_numpy_bits(g) for g in grads]
+    want, want_seed, counts = orc.filter_any_seed(np_grads, tau)
+    g_seed = int(seed.cpu().item())
+    g_mask = mask.cpu().numpy()
+    order = [(g_seed + t) % K for t in range(K)]
+    r, replays = oracle_with_replay(np_grads, tau, order, g_mask)
+    if replays == 0:
+        assert g_seed == want_seed, (g_seed, want_seed, counts.tolist())
+    assert int(count.cpu().item()) == r.count and g_mask.tolist() == r.mask.tolist()
+    assert r.count >= int(counts.max()) - replays
+    g_dist = dist.cpu().numpy().astype(np.float64)
+    assert float(np.max(np.abs(g_dist - r.dist))) <= DIST_ATOL
+    assert rel_l2(macro.cpu().numpy(), r.out) <= MACRO_RTOL[grads[0].dtype]
+    # bit-identical to the plain filter run in the winning order
+    plain = gaf.gaf_filter_accumulate(grads, tau, workspace, order=order)
+    assert torch.equal(plain[0], macro) and torch.equal(plain[1], mask)
+    return {"seed": g_seed, "count": r.count, "counts": counts.tolist()}

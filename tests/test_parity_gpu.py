@@ -8,7 +8,7 @@ import torch
 
 import paper_2412_18052_b200 as gaf
 from paper_2412_18052_b200 import workloads
-from parity import check_cosdist, check_filter, check_pairwise
+from parity import check_any_seed, check_cosdist, check_filter, check_pairwise
 
 pytestmark = pytest.mark.gpu
 
@@ -198,6 +198,29 @@ def test_filter_host_entry_point(ws):
     macro, mask, dist, count = gaf.gaf_filter_accumulate(w.grads, 0.8, ws)
     assert torch.equal(macro.cpu(), macro_h) and torch.equal(mask.cpu(), mask_h)
     assert torch.equal(dist.cpu(), dist_h) and int(count.item()) == int(count_h.item())
+
+
+# ---------------------------------------- order-indifferent variant (Section 3.1) --
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_any_seed_variant(ws, dtype):
+    # the paper's degenerate case: a first gradient orthogonal to all the others
+    D = 70_001
+    base = torch.randn(D, device="cuda") * 1e-3
+    odd = torch.zeros(D, device="cuda"); odd[::2] = 1e-3
+    odd = odd - (odd @ base) / (base @ base) * base                 # orthogonal to base
+    gs = [odd] + [base + 0.3 * torch.randn(D, device="cuda") * 1e-3 for _ in range(3)]
+    if dtype == "bf16":
+        gs = [g.to(torch.bfloat16) for g in gs]
+    macro, mask, dist, count, *_ = gaf.gaf_filter_accumulate(gs, 0.5, ws)
+    assert int(count.item()) == 1                                    # plain Algorithm 1 wastes the macrobatch
+    r = check_any_seed(gs, 0.5, ws)
+    assert r["seed"] == 1 and r["count"] == 3
+    # mixtures over every Gram path: K <= 8, tensor cores (bf16, K <= 32), tiled (the rest)
+    for K, Dk in ((1, 1000), (2, 5003), (5, 300_007), (8, 1_000_001), (12, 400_003), (32, 200_001), (40, 50_001)):
+        w = _mix(K, Dk, dtype, seed=900 + K)
+        r = check_any_seed(w.grads, 0.97, ws)
+        assert r["count"] == max(r["counts"])
 
 
 # ------------------------------------------------- the named configurations --
