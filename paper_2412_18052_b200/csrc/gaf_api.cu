@@ -190,8 +190,17 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     for (int t = 0; t < K; ++t) m.g[t] = g[ord[t]];
     m.K = K; m.D = D; m.out = macro_out; m.ctl = ctl;
     const int grid = stream_grid(D, kMsThreads, sms);
-    masked_mean_kernel<T><<<grid, kMsThreads, 0, st>>>(m);
+    // programmatic dependent launch: the blocks may be placed while the Gram pass winds down
+    // (its last CTA is still totalling partials); the kernel itself waits for that grid
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kMsThreads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, masked_mean_kernel<T>, m);
     ++g_launches;
+    if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }
 

@@ -267,6 +267,10 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
             for (int c = r; c < KT; ++c, ++p) acc[p] = fmaf(x[r], x[c], acc[p]);
     }
     flush();
+    // the streaming part of this CTA is over: a kernel launched as a programmatic dependent
+    // (the masked-mean pass) may start occupying SMs; it still waits for this whole grid
+    // before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __syncthreads();
     if (threadIdx.x < NP) {
         double s = 0.0;
@@ -366,6 +370,9 @@ __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid
     __shared__ const T *list[GAF_MAX_K];
     __shared__ int n_list;
     __shared__ float cdiv_s;
+    // when launched as a programmatic dependent of the Gram pass: wait until that grid has
+    // completed and its writes (the accept bits) are visible; otherwise a no-op
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (threadIdx.x == 0) {
         const unsigned long long bits = *reinterpret_cast<const volatile unsigned long long *>(&a.ctl->accept_bits);
         const int seed = *reinterpret_cast<const volatile int *>(&a.ctl->ring_seed);
