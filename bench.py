@@ -197,20 +197,50 @@ def time_oracle(cfg: int, tau: float, seconds: float):
     return gbs, per_call, sample
 
 
+def workload_label(cfg, K, D, dtype, tau):
+    return (f"configuration {cfg}: K={K}, D={D}, {dtype} inputs, tau={tau}, shared+private Gaussian mixture" +
+            (" with ResNet18 per-tensor scales" if cfg == 2 else ""))
+
+
 def run_reference(args):
+    """Reference arm: the CPU oracle as it stands, one thread, W warm-up + K timed steps.
+    A step is one whole oracle call on a bounded sample of the workload: the same recipe at a
+    D chosen so that the run ends within about two minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    steps = max(1, args.steps)
-    # each "step" of this arm is one oracle call on the bounded sample
-    budget = min(120.0, max(5.0, args.cpu_seconds))
-    gbs, per_call, sample = time_oracle(args.workload, args.tau, budget)
+    from oracle import gaf_oracle as orc
+    from paper_2412_18052_b200 import workloads
+
+    cfg = 2 if args.workload == 3 else args.workload
+    full = {1: 1_000_000, 2: workloads.RESNET18_100_NUMEL, 4: workloads.GPT2_SMALL_NUMEL, 5: 1_000_000_000}[cfg]
+    K = {1: 4, 2: 4, 4: 8, 5: 8}[cfg]
+    b = 2 if cfg == 5 else 4
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    # about 2.2 GB/s of gradient bytes on one core: size the sample for ~100 s in all
+    budget_s = 100.0
+    d_fit = int(budget_s / (steps + warmup) * 2.0e9 / (K * b))
+    D = max(50_000, min(full, d_fit))
+    w = workloads.config(cfg, device="cpu", D=None if D == full else D)
+    grads = [workloads.as_numpy_bits(g) for g in w.grads]
+    for _ in range(warmup):
+        orc.filter_accumulate(grads, args.tau)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        orc.filter_accumulate(grads, args.tau)
+    dt = time.perf_counter() - t0
+    per_call = dt / steps
+    gbs = w.K * w.elem_bytes * w.D / per_call / 1e9
+    sample = (f"configuration {cfg} recipe, K={w.K}, D={w.D:,} {w.dtype}"
+              f"{'' if D == full else ' (reduced from D=%d)' % full}, one oracle call per step, "
+              f"{steps} steps, {dt:.1f} s of CPU work")
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": steps, "warmup": args.warmup, "ms_per_step": per_call * 1e3,
+        "steps": steps, "warmup": warmup, "ms_per_step": per_call * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": f"configuration {args.workload}", "tau": args.tau},
+        "config": {"workload": workload_label(cfg, K, full, w.dtype, args.tau), "K": K, "D": full,
+                   "input_dtype": w.dtype, "tau": args.tau, "sample_D": w.D},
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -422,9 +452,7 @@ def run_ours(args):
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
-                "workload": f"configuration {cfg}: K={K}, D={D}, {w0.dtype} inputs, tau={args.tau}, "
-                            f"shared+private Gaussian mixture" +
-                            (" with ResNet18 per-tensor scales" if cfg == 2 else ""),
+                "workload": workload_label(cfg, K, D, w0.dtype, args.tau),
                 "K": K, "D": D, "input_dtype": w0.dtype, "tau": args.tau,
                 "schedule": {0: "auto", 1: "stepwise", 2: "gram-first"}[args.schedule] +
                             (" -> " + {1: "stepwise", 2: "gram-first"}[sched_used] if not args.schedule else ""),
