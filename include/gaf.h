@@ -171,6 +171,28 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Streaming form of Algorithm 1, for micro-gradients that arrive one at a time (as
+ * they do around a ring, Section 1 / Section 3.1): the loop body of Algorithm 1 per
+ * call.  The state lives in `workspace` (one stream of calls per workspace) and in
+ * the caller's running-sum buffer `acc` (D floats, 16-byte aligned).
+ *   gaf_stream_begin   g <- seed; c <- 1
+ *   gaf_stream_push    gradient number t (t = 1, 2, ... in arrival order, t < GAF_MAX_K):
+ *                      D_c(g_t, g) by Eq. 4; if <= tau: g <- g + g_t, c <- c + 1.
+ *                      `g` may be reused as soon as the call's work on the stream is done.
+ *   gaf_stream_end     acc <- g / c (Eq. 5); mask_out[K], dist_out[K] (may be NULL) in
+ *                      ARRIVAL order (entry 0 = seed: 1 and 0), count_out = c
+ * Same arithmetic as gaf_filter_accumulate with GAF_SCHED_STEPWISE: the result is
+ * bit-identical to that call on the same gradients in arrival order.
+ */
+int gaf_stream_begin(const void *seed, int64_t D, int dtype, float *acc,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+int gaf_stream_push(const void *g, int t, int64_t D, int dtype, double tau, float *acc,
+                    void *workspace, size_t workspace_bytes, void *cuda_stream);
+int gaf_stream_end(int K, int64_t D, float *acc, uint8_t *mask_out, float *dist_out,
+                   int32_t *count_out,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The same operation for gradients that live in HOST memory (pinned memory
  * makes the copies asynchronous and fast).  Copies each gradient to the device
  * staging area, runs gaf_filter_accumulate, copies the results back and

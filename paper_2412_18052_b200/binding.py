@@ -24,7 +24,7 @@ EXPORTS = [
     "gaf_error_string", "gaf_workspace_bytes", "gaf_workspace_init", "gaf_cosdist",
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
     "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
-    "gaf_filter_accumulate_any_seed",
+    "gaf_filter_accumulate_any_seed", "gaf_stream_begin", "gaf_stream_push", "gaf_stream_end",
 ]
 
 
@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.gaf_last_launch_count.argtypes = []
         L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.gaf_filter_accumulate_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gaf_stream_begin.argtypes = [vp, i64, i32, vp, vp, sz, vp]
+        L.gaf_stream_push.argtypes = [vp, i32, i64, i32, dbl, vp, vp, sz, vp]
+        L.gaf_stream_end.argtypes = [i32, i64, vp, vp, vp, vp, vp, sz, vp]
         for name in EXPORTS:
             if name != "gaf_error_string":
                 getattr(L, name).restype = i32
@@ -196,6 +199,30 @@ def gaf_filter_accumulate_any_seed(grads: Sequence[torch.Tensor], tau: float, wo
         seed_out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
         "gaf_filter_accumulate_any_seed")
     return macro_out, mask_out, dist_out, count_out, seed_out
+
+
+def gaf_stream_begin(seed: torch.Tensor, acc: torch.Tensor, workspace: torch.Tensor) -> None:
+    """Streaming form: g <- seed, c <- 1 (``acc`` is the caller's float32 running sum)."""
+    _check(lib().gaf_stream_begin(seed.data_ptr(), seed.numel(), _dtype_code(seed), acc.data_ptr(),
+                                  workspace.data_ptr(), workspace.numel(), _stream()), "gaf_stream_begin")
+
+
+def gaf_stream_push(g: torch.Tensor, t: int, tau: float, acc: torch.Tensor, workspace: torch.Tensor) -> None:
+    """Streaming form: test gradient number t (arrival order, from 1) and add it if accepted."""
+    _check(lib().gaf_stream_push(g.data_ptr(), int(t), g.numel(), _dtype_code(g), float(tau), acc.data_ptr(),
+                                 workspace.data_ptr(), workspace.numel(), _stream()), "gaf_stream_push")
+
+
+def gaf_stream_end(K: int, acc: torch.Tensor, workspace: torch.Tensor):
+    """Streaming form: acc <- g / c.  Returns (mask[K], dist[K], count) in arrival order."""
+    dev = acc.device
+    mask = torch.empty(K, dtype=torch.uint8, device=dev)
+    dist = torch.empty(K, dtype=torch.float32, device=dev)
+    count = torch.empty(1, dtype=torch.int32, device=dev)
+    _check(lib().gaf_stream_end(int(K), acc.numel(), acc.data_ptr(), mask.data_ptr(), dist.data_ptr(),
+                                count.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
+           "gaf_stream_end")
+    return mask, dist, count
 
 
 def gaf_filter_accumulate_host(grads_host: Sequence[torch.Tensor], tau: float,

@@ -11,6 +11,7 @@
 #include "gaf_gramfilter.cuh"
 #include "gaf_pairwise.cuh"
 #include "gaf_stepwise.cuh"
+#include "gaf_stream.cuh"
 
 namespace {
 
@@ -403,6 +404,76 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
                                    seed_out, base, di.sms, di.l2_bytes, st)
         : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
                                            count_out, seed_out, base, di.sms, di.l2_bytes, st);
+}
+
+int gaf_stream_begin(const void *seed, int64_t D, int dtype, float *acc, void *workspace,
+                     size_t workspace_bytes, void *cuda_stream) {
+    g_launches = 0;
+    if ((!seed && D > 0) || (!acc && D > 0) || D < 0) return GAF_ERR_ARG;
+    if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
+    if (!aligned16(seed) || !aligned16(acc)) return GAF_ERR_ALIGN;
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    Control *ctl = reinterpret_cast<Control *>(base);
+    // g <- seed, c <- 1: the one-gradient form of the stepwise kernel (its mask, distance and
+    // count outputs go to the control block)
+    StepArgs a{};
+    a.acc = acc; a.D = D; a.ctl = ctl; a.partials = reinterpret_cast<double *>(base + kPartialsOffset);
+    a.g_seed = seed; a.seed_index = 0; a.K = 1;
+    a.mask_out = ctl->stream_mask; a.dist_out = ctl->stream_dist; a.count_out = &ctl->count;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int grid = stream_grid(D, kStepThreads, di.sms);
+    if (dtype == GAF_F32) step_kernel<float, kOnly><<<grid, kStepThreads, 0, st>>>(a);
+    else step_kernel<__nv_bfloat16, kOnly><<<grid, kStepThreads, 0, st>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int gaf_stream_push(const void *g, int t, int64_t D, int dtype, double tau, float *acc, void *workspace,
+                    size_t workspace_bytes, void *cuda_stream) {
+    g_launches = 0;
+    if ((!g && D > 0) || (!acc && D > 0) || D < 0 || t < 1 || t >= GAF_MAX_K || tau != tau) return GAF_ERR_ARG;
+    if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
+    if (!aligned16(g) || !aligned16(acc)) return GAF_ERR_ALIGN;
+    {
+        const uintptr_t o0 = reinterpret_cast<uintptr_t>(acc), o1 = o0 + size_t(D) * 4;
+        const uintptr_t g0 = reinterpret_cast<uintptr_t>(g), g1 = g0 + size_t(D) * elem_bytes(dtype);
+        if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
+    }
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    StreamArgs a{g, acc, D, reinterpret_cast<Control *>(base),
+                 reinterpret_cast<double *>(base + kPartialsOffset), tau, t};
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int grid = stream_grid(D, kStreamThreads, di.sms);
+    if (dtype == GAF_F32) {
+        stream_test_kernel<float><<<grid, kStreamThreads, 0, st>>>(a);
+        stream_add_kernel<float><<<grid, kStreamThreads, 0, st>>>(a);
+    } else {
+        stream_test_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, st>>>(a);
+        stream_add_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, st>>>(a);
+    }
+    g_launches += 2;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+int gaf_stream_end(int K, int64_t D, float *acc, uint8_t *mask_out, float *dist_out, int32_t *count_out,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    g_launches = 0;
+    if (K < 1 || K > GAF_MAX_K || D < 0 || (!acc && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
+    if (!aligned16(acc)) return GAF_ERR_ALIGN;
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    StreamEndArgs a{acc, D, K, static_cast<const Control *>(workspace), mask_out, dist_out, count_out};
+    const int grid = stream_grid(D, kStreamThreads, di.sms);
+    stream_end_kernel<<<grid, kStreamThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }
 
 int gaf_host_staging_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {

@@ -25,6 +25,8 @@ struct Control {
     unsigned long long accept_bits;     // Gram-first schedule: bit t set = step t accepted
     int decision[GAF_MAX_K];            // by step t: 1 accept, 0 reject
     double sums[GAF_MAX_K][3];          // by step t: {g_i.g, |g|^2, |g_i|^2}
+    float stream_dist[GAF_MAX_K];       // streaming form: distance of arrival t
+    uint8_t stream_mask[GAF_MAX_K];     // streaming form: decision of arrival t
 };
 constexpr size_t kControlBytes = 4096;  // sizeof(Control) rounded up
 static_assert(sizeof(Control) <= kControlBytes, "control block");

@@ -200,6 +200,28 @@ def test_filter_host_entry_point(ws):
     assert torch.equal(dist.cpu(), dist_h) and int(count.item()) == int(count_h.item())
 
 
+# ------------------------------------------------------------ streaming form --
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_streaming_form_matches_oracle_and_batch_call(ws, dtype):
+    from oracle import gaf_oracle as orc
+    for K, D, tau in ((1, 1001, 0.97), (2, 8, 0.97), (4, 300_007, 0.6), (7, 1_000_003, 0.97)):
+        w = _mix(K, D, dtype, seed=700 + K)
+        acc = torch.empty(D, dtype=torch.float32, device="cuda")
+        gaf.gaf_stream_begin(w.grads[0], acc, ws)
+        for t in range(1, K):
+            gaf.gaf_stream_push(w.grads[t], t, tau, acc, ws)
+        mask, dist, count = gaf.gaf_stream_end(K, acc, ws)
+        assert gaf.gaf_read_status(ws) == 0
+        want = orc.filter_accumulate([workloads.as_numpy_bits(g) for g in w.grads], tau)
+        assert mask.cpu().numpy().tolist() == want.mask.tolist() and int(count.item()) == want.count
+        assert float(np.max(np.abs(dist.cpu().numpy() - want.dist))) < 1e-5
+        got = acc.cpu().numpy().astype(np.float64)
+        assert float(np.linalg.norm(got - want.out) / np.linalg.norm(want.out)) < (1e-6 if dtype == "f32" else 1e-3)
+        batch = gaf.gaf_filter_accumulate(w.grads, tau, ws, schedule=gaf.GAF_SCHED_STEPWISE)
+        assert torch.equal(batch[0], acc) and torch.equal(batch[1], mask) and torch.equal(batch[2], dist)
+
+
 # ---------------------------------------- order-indifferent variant (Section 3.1) --
 
 @pytest.mark.parametrize("dtype", DTYPES)
