@@ -148,11 +148,20 @@ __device__ __forceinline__ Sums3 block_reduce(Sums3 s, double *scratch) {
 __device__ __forceinline__ Sums3 warp_sum_partials(const double *partials, int n) {
     const int lane = threadIdx.x & 31;
     Sums3 s = {0.0, 0.0, 0.0};
-#pragma unroll 4
-    for (int i = lane; i < n; i += 32) {
-        const double a = __ldcg(partials + 3 * i), b = __ldcg(partials + 3 * i + 1),
-                     c = __ldcg(partials + 3 * i + 2);
-        s.p += a; s.na += b; s.ng += c;
+    // batches of 10 entries per lane (320 CTAs) whose loads are all issued before the first add:
+    // this runs on the serial tail of a launch, one L2 round trip per batch
+    for (int base = 0; base < n; base += 320) {
+        double a[10], b[10], c[10];
+#pragma unroll
+        for (int k = 0; k < 10; ++k) {
+            const int i = base + lane + 32 * k;
+            const bool ok = i < n;
+            a[k] = ok ? __ldcg(partials + 3 * i) : 0.0;
+            b[k] = ok ? __ldcg(partials + 3 * i + 1) : 0.0;
+            c[k] = ok ? __ldcg(partials + 3 * i + 2) : 0.0;
+        }
+#pragma unroll
+        for (int k = 0; k < 10; ++k) { s.p += a[k]; s.na += b[k]; s.ng += c[k]; }
     }
     return warp_reduce(s);
 }

@@ -35,16 +35,20 @@ struct ReplayArgs {
 };
 
 // Algorithm 1 on the Gram matrix (indexed by processing step): one thread.
-// gram is K x K row-major in binary64.
-__device__ __forceinline__ void replay_on_gram(const ReplayArgs &r, const volatile double *gram) {
+// gram is K x K row-major in binary64.  With `publish` the decisions, distances and count go
+// to the outputs and the control block; the accept bits (bit t = step t) are returned either way.
+__device__ __forceinline__ unsigned long long replay_on_gram(const ReplayArgs &r, const volatile double *gram,
+                                                             bool publish) {
     const int K = r.K;
     Control *c = r.ctl;
     int status = 0, count = 1;
-    unsigned long long bits = 1ull;         // bit t set = step t accepted (step 0 is the seed)
+    unsigned long long bits = 1ull;         // step 0 is the seed
     double na = gram[0];                    // |g|^2 of the running sum
-    c->decision[0] = 1;
-    r.mask_out[r.idx[0]] = 1;
-    if (r.dist_out) r.dist_out[r.idx[0]] = 0.0f;
+    if (publish) {
+        c->decision[0] = 1;
+        r.mask_out[r.idx[0]] = 1;
+        if (r.dist_out) r.dist_out[r.idx[0]] = 0.0f;
+    }
     for (int t = 1; t < K; ++t) {
         double p = 0.0;                     // <g_t, running sum>
         for (int u = 0; u < t; ++u)
@@ -52,22 +56,26 @@ __device__ __forceinline__ void replay_on_gram(const ReplayArgs &r, const volati
         const double ng = gram[(size_t)t * K + t];
         const double d = cosine_distance(p, na, ng, &status);
         const int accept = (d <= r.tau) ? 1 : 0;
-        c->decision[t] = accept;
-        c->sums[t][0] = p; c->sums[t][1] = na; c->sums[t][2] = ng;
-        r.mask_out[r.idx[t]] = (uint8_t)accept;
-        if (r.dist_out) r.dist_out[r.idx[t]] = (float)d;
+        if (publish) {
+            c->decision[t] = accept;
+            c->sums[t][0] = p; c->sums[t][1] = na; c->sums[t][2] = ng;
+            r.mask_out[r.idx[t]] = (uint8_t)accept;
+            if (r.dist_out) r.dist_out[r.idx[t]] = (float)d;
+        }
         if (accept) {
             bits |= 1ull << t;
             na = na + 2.0 * p + ng;         // |g + g_t|^2
             ++count;
         }
     }
-    c->accept_bits = bits;
-    c->ring_seed = -1;
-    c->count = count;
-    c->status = status;
-    *r.count_out = count;
-    __threadfence();
+    if (publish) {
+        c->accept_bits = bits;
+        c->ring_seed = -1;
+        c->count = count;
+        c->status = status;
+        *r.count_out = count;
+    }
+    return bits;
 }
 
 // Order-indifferent variant (end of Section 3.1): Algorithm 1 from every seed s with the
@@ -287,12 +295,21 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     if (!is_last) return;
     __threadfence();
 
-    // last CTA: fixed-order totals (one warp per pair), then the scalar walk
+    // last CTA: fixed-order totals (one warp per pair; all of a lane's loads are issued together,
+    // this is the serial tail of the call), then the scalar walk out of shared memory
+    __shared__ double sgram[KT * KT];
     const double *part = a.partials;
+    constexpr int kRounds = (kGsMaxCtas + 31) / 32;
     for (int p = warp; p < NP; p += kGsThreads / 32) {
+        double v[kRounds];
+#pragma unroll
+        for (int k = 0; k < kRounds; ++k) {
+            const int i = lane + 32 * k;
+            v[k] = i < (int)gridDim.x ? __ldcg(part + (size_t)i * 64 + p) : 0.0;
+        }
         double s = 0.0;
-#pragma unroll 4
-        for (int i = lane; i < (int)gridDim.x; i += 32) s += __ldcg(part + (size_t)i * 64 + p);
+#pragma unroll
+        for (int k = 0; k < kRounds; ++k) s += v[k];
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) s += shfl_down_f64(s, d);
         if (lane == 0) {
@@ -300,27 +317,27 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
             int r = 0, rem = p;
             while (rem >= KT - r) { rem -= KT - r; ++r; }
             const int c = r + rem;
+            sgram[r * KT + c] = s;
+            sgram[c * KT + r] = s;
             a.gram[r * KT + c] = s;
             a.gram[c * KT + r] = s;
         }
     }
-    __threadfence();
     __syncthreads();
     if (a.ring.K > 0) {
         __shared__ int ring_count[kGsMaxK];
         __shared__ unsigned long long ring_bits[kGsMaxK];
-        ring_replay_on_gram(a.ring, a.gram, ring_count, ring_bits);
+        ring_replay_on_gram(a.ring, sgram, ring_count, ring_bits);
         return;
     }
     if (a.pair_dist_out == nullptr) {
-        if (threadIdx.x == 0) replay_on_gram(a.replay, a.gram);
+        if (threadIdx.x == 0) { replay_on_gram(a.replay, sgram, true); __threadfence(); }
         return;
     }
     // pairwise mode: Eq. 4 for every pair
     if (threadIdx.x < KT * KT) {
-        const volatile double *G = a.gram;
         const int i = threadIdx.x / KT, j = threadIdx.x % KT;
-        const double gii = G[i * KT + i], gjj = G[j * KT + j], gij = G[threadIdx.x];
+        const double gii = sgram[i * KT + i], gjj = sgram[j * KT + j], gij = sgram[threadIdx.x];
         int status = 0;
         const double d = (i == j && gii > 0.0) ? 0.0 : cosine_distance(gij, gii, gjj, &status);
         a.pair_dist_out[threadIdx.x] = (float)d;
@@ -339,7 +356,7 @@ __global__ void gram_replay_kernel(ReplayArgs r, const double *gram_by_index, do
     }
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) replay_on_gram(r, gram_by_step);
+    if (threadIdx.x == 0) { replay_on_gram(r, gram_by_step, true); __threadfence(); }
 }
 
 // Any-seed walk as its own launch (Gram matrix by original index from the tiled or
@@ -373,9 +390,13 @@ __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid
     // when launched as a programmatic dependent of the Gram pass: wait until that grid has
     // completed and its writes (the accept bits) are visible; otherwise a no-op
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    unsigned long long bits = 0;
+    int seed = -1;
     if (threadIdx.x == 0) {
-        const unsigned long long bits = *reinterpret_cast<const volatile unsigned long long *>(&a.ctl->accept_bits);
-        const int seed = *reinterpret_cast<const volatile int *>(&a.ctl->ring_seed);
+        bits = __ldcg(&a.ctl->accept_bits);                      // (two independent L2 loads)
+        seed = __ldcg(&a.ctl->ring_seed);
+    }
+    if (threadIdx.x == 0) {
         const int start = seed < 0 ? 0 : seed;
         int n = 0;
         for (int t = 0; t < a.K; ++t) {
