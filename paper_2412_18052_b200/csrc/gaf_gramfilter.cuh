@@ -369,6 +369,33 @@ __global__ void gram_ring_replay_kernel(RingArgs r, const double *gram_by_index)
 
 // ------------------------------------------------------- masked mean (Eq. 5) --
 
+// Eight consecutive elements as loaded (streaming, evict-first), widened on use.
+template <typename T> struct RawOct;
+template <> struct RawOct<float> {
+    float4 a, b;
+    static __device__ __forceinline__ RawOct load(const float *base, int64_t e) {
+        const float4 *p = reinterpret_cast<const float4 *>(base + e);
+        return {__ldcs(p), __ldcs(p + 1)};
+    }
+    __device__ __forceinline__ void widen(float (&v)[8]) const {
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+};
+template <> struct RawOct<__nv_bfloat16> {
+    uint4 r;
+    static __device__ __forceinline__ RawOct load(const __nv_bfloat16 *base, int64_t e) {
+        return {__ldcs(reinterpret_cast<const uint4 *>(base + e))};
+    }
+    __device__ __forceinline__ void widen(float (&v)[8]) const {
+        const unsigned int w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[2 * k] = bf16_bits_to_float(w[k] & 0xFFFFu);
+            v[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        }
+    }
+};
+
 struct MaskedMeanArgs {
     const void *g[GAF_MAX_K];               // processing order; original order in any-seed mode, where
                                             // the order starts at the winning seed and wraps around
@@ -411,25 +438,50 @@ __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid
     const float cdiv = cdiv_s;
     const int64_t n_oct = a.D / kOct;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < n_oct; o += stride) {
-        const int64_t e = (n_oct - 1 - o) * kOct;
-        float v[8];
-        load8_stream<T>(list[0], e, v);
-        for (int i = 1; i < n; i += 4) {
-            float w[4][8];
+    // U groups of 8 elements per thread and round (two for 2-byte inputs, so that as many bytes
+    // are in flight as with 4-byte inputs); loads stay packed until they are added
+    constexpr int U = sizeof(T) == 2 ? 2 : 1;
+    constexpr int kChunk = 3;                       // further gradients fetched together
+    for (int64_t o0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o0 < n_oct; o0 += stride * U) {
+        int64_t e[U];
+        bool ok[U];
+        RawOct<T> first[U];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (i + u < n) load8_stream<T>(list[i + u], e, w[u]);
+        for (int u = 0; u < U; ++u) {
+            const int64_t o = o0 + u * stride;
+            ok[u] = o < n_oct;
+            e[u] = (n_oct - 1 - (ok[u] ? o : 0)) * kOct;
+            if (ok[u]) first[u] = RawOct<T>::load(list[0], e[u]);
+        }
+        float v[U][8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (i + u < n) {
+        for (int u = 0; u < U; ++u)
+            if (ok[u]) first[u].widen(v[u]);
+        for (int i = 1; i < n; i += kChunk) {
+            RawOct<T> w[U][kChunk];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) v[k] += w[u][k];
-                }
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j)
+                    if (ok[u] && i + j < n) w[u][j] = RawOct<T>::load(list[i + j], e[u]);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int j = 0; j < kChunk; ++j)
+                    if (ok[u] && i + j < n) {
+                        float x[8];
+                        w[u][j].widen(x);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) v[u][k] += x[k];
+                    }
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) v[k] = v[k] / cdiv;
-        store8(a.out, e, v, true);
+        for (int u = 0; u < U; ++u)
+            if (ok[u]) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[u][k] = v[u][k] / cdiv;
+                store8(a.out, e[u], v[u], true);
+            }
     }
     const int64_t tail0 = n_oct * kOct;
     if (blockIdx.x == 0 && tail0 + threadIdx.x < a.D) {
