@@ -200,6 +200,34 @@ def test_filter_host_entry_point(ws):
     assert torch.equal(dist.cpu(), dist_h) and int(count.item()) == int(count_h.item())
 
 
+def test_filter_random_cases(ws):
+    """Seeded random shapes, thresholds, orders and schedules against the oracle."""
+    rng = np.random.RandomState(2024)
+    for case in range(48):
+        K = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 13, 16, 31, 32, 33, 40]))
+        D = int(rng.choice([0, 1, 7, 63, 1000, 4099, 65_537, 300_001, 1_048_576 + 3]))
+        if K > 16:
+            D = min(D, 65_537)
+        dtype = "bf16" if rng.rand() < 0.5 else "f32"
+        tau = float(rng.choice([0.3, 0.8, 0.97, 1.0, 1.1, 1.6]))
+        order = [int(x) for x in rng.permutation(K)] if rng.rand() < 0.5 else None
+        schedule = int(rng.choice([gaf.GAF_SCHED_AUTO, gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_GRAM]))
+        w = _mix(K, D, dtype, seed=5000 + case, sigma=float(rng.choice([1e-3, 1.0, 30.0])))
+        check_filter(w.grads, tau, ws, order=order, schedule=schedule, expect_status=None)
+
+
+def test_filter_partly_cancelling_gradients(ws):
+    """Accepted gradients that nearly cancel: the norm of the running sum is a small
+    difference of large Gram entries in the Gram-first schedule."""
+    D = 200_003
+    g = torch.randn(D, device="cuda") * 1e-3
+    gs = [g, -0.99 * g + 1e-6 * torch.randn(D, device="cuda"), torch.randn(D, device="cuda") * 1e-3,
+          0.5 * g + 1e-4 * torch.randn(D, device="cuda")]
+    for schedule in SCHEDULES:
+        check_filter(gs, 2.0, ws, schedule=schedule)
+        check_filter(gs, 1.2, ws, schedule=schedule)
+
+
 # ------------------------------------------------------------ streaming form --
 
 @pytest.mark.parametrize("dtype", DTYPES)
