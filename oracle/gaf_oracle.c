@@ -181,6 +181,37 @@ int gaf_oracle_filter_any_seed(const void *const *grads, int K, int64_t D, int d
 }
 
 /*
+ * Bucketed variant (Section 5 notes that inside a ring all-reduce the cosine distance
+ * would have to be applied "to buckets at a time"): the D parameters are cut into S
+ * consecutive buckets, bucket b = elements [offsets[b], offsets[b+1]), and Algorithm 1
+ * followed by Eq. 5 runs on every bucket independently -- its own running sum, its own
+ * decisions, its own count.                                     [parity unpinned]
+ *   offsets  S+1 ascending element offsets, offsets[0] = 0, offsets[S] = D
+ *   g        D doubles: per-bucket g/c on return
+ *   mask     S*K bytes, row b = bucket b, by original index
+ *   dist     S*K doubles;  count  S entries
+ */
+int gaf_oracle_filter_bucketed(const void *const *grads, int K, int64_t D, int dtype,
+                               double tau, const int32_t *order, int S,
+                               const int64_t *offsets, double *g, uint8_t *mask,
+                               double *dist, int32_t *count)
+{
+    if (K < 1 || K > 4096 || S < 1 || offsets[0] != 0 || offsets[S] != D) return 1;
+    size_t esize = dtype == ORACLE_F32 ? 4 : 2;
+    const void *sub[4096];
+    for (int b = 0; b < S; ++b) {
+        int64_t lo = offsets[b], hi = offsets[b + 1];
+        if (hi < lo) return 1;
+        for (int i = 0; i < K; ++i) sub[i] = (const char *)grads[i] + (size_t)lo * esize;
+        int rc = gaf_oracle_filter_accumulate(sub, K, hi - lo, dtype, tau, order, NULL, g + lo,
+                                              mask + (size_t)b * K, dist + (size_t)b * K,
+                                              count + b, NULL);
+        if (rc) return rc;
+    }
+    return 0;
+}
+
+/*
  * Pairwise cosine distances between K micro-gradients (the quantity the
  * paper's cosine-distance figures plot).  gram and dist are K*K row-major.
  * Diagonal: 0 when the norm is non-zero; rows/columns of a zero-norm vector

@@ -66,6 +66,8 @@ def _load():
         lib.gaf_oracle_filter_accumulate.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, vp]
         lib.gaf_oracle_filter_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, vp]
         lib.gaf_oracle_filter_any_seed.restype = ctypes.c_int
+        lib.gaf_oracle_filter_bucketed.argtypes = [vp, i32, i64, i32, dbl, vp, i32, vp, vp, vp, vp, vp]
+        lib.gaf_oracle_filter_bucketed.restype = ctypes.c_int
         lib.gaf_oracle_pairwise.argtypes = [vp, i32, i64, i32, vp, vp]
         lib.gaf_oracle_plain_average.argtypes = [vp, i32, i64, i32, vp]
         for f in (lib.gaf_oracle_cosdist, lib.gaf_oracle_filter_accumulate,
@@ -174,6 +176,28 @@ def filter_any_seed(grads: Sequence[np.ndarray], tau: float):
         raise ValueError("oracle rejected its arguments")
     res = FilterResult(out, mask, dist, int(count.value), np.zeros((K, 3)))
     return res, int(seed.value), counts
+
+
+def filter_bucketed(grads: Sequence[np.ndarray], tau: float, offsets: Sequence[int],
+                    order: Optional[Sequence[int]] = None):
+    """Bucketed variant: Algorithm 1 + Eq. 5 independently on every bucket
+    [offsets[b], offsets[b+1]).  Returns (out[D], mask[S,K], dist[S,K], count[S])."""
+    arrs, ptrs, code, D = _prep(grads)
+    K = len(arrs)
+    off = np.ascontiguousarray(offsets, dtype=np.int64)
+    S = off.size - 1
+    order_arr = None if order is None else np.ascontiguousarray(order, dtype=np.int32)
+    out = np.empty(D, dtype=np.float64)
+    mask = np.zeros((S, K), dtype=np.uint8)
+    dist = np.zeros((S, K), dtype=np.float64)
+    count = np.zeros(S, dtype=np.int32)
+    rc = _load().gaf_oracle_filter_bucketed(
+        ctypes.cast(ptrs, ctypes.c_void_p), K, D, code, float(tau),
+        None if order_arr is None else order_arr.ctypes.data, S, off.ctypes.data,
+        out.ctypes.data, mask.ctypes.data, dist.ctypes.data, count.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle rejected its arguments")
+    return out, mask, dist, count
 
 
 def pairwise_cosdist(grads: Sequence[np.ndarray]):

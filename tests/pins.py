@@ -396,6 +396,30 @@ def pin_any_seed_variant():
         assert np.array_equal(r.out, per_seed[best].out) and np.array_equal(r.dist, per_seed[best].dist)
 
 
+def pin_bucketed_variant():
+    """Bucketed variant: one bucket is plain GAF; several buckets are plain GAF on each slice;
+    an empty bucket is legal; buckets decide independently."""
+    rng = np.random.RandomState(13)
+    K, D = 4, 60
+    gs = _rand_grads(rng, K, D, "f32", shared=0.6)
+    gs[2][:20] = -gs[0][:20]                       # disagrees in the first bucket only
+    whole = orc.filter_accumulate(gs, 0.9)
+    out, mask, dist, count = orc.filter_bucketed(gs, 0.9, [0, D])
+    assert np.array_equal(out, whole.out) and mask[0].tolist() == whole.mask.tolist()
+    assert count.tolist() == [whole.count] and np.array_equal(dist[0], whole.dist)
+    offsets = [0, 20, 20, 47, D]
+    out, mask, dist, count = orc.filter_bucketed(gs, 0.9, offsets, order=[1, 0, 3, 2])
+    seen = set()
+    for b in range(4):
+        lo, hi = offsets[b], offsets[b + 1]
+        r = orc.filter_accumulate([g[lo:hi] for g in gs], 0.9, order=[1, 0, 3, 2])
+        assert np.array_equal(out[lo:hi], r.out) and mask[b].tolist() == r.mask.tolist()
+        assert count[b] == r.count and np.array_equal(dist[b], r.dist)
+        seen.add(tuple(mask[b].tolist()))
+    assert mask[1].tolist() == [0, 1, 0, 0] and count[1] == 1   # empty bucket: zero norms, distance 1 > tau
+    assert len(seen) >= 2                           # buckets really decide on their own
+
+
 ALL_PINS = [
     pin_stated_values,
     pin_figure2_angles,
@@ -413,4 +437,5 @@ ALL_PINS = [
     pin_forced_decisions,
     pin_closed_form_mixture,
     pin_any_seed_variant,
+    pin_bucketed_variant,
 ]

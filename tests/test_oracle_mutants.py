@@ -39,6 +39,9 @@ MUTANTS = [
     ("pairwise_wrong_norm", "gram[i * K + i], gram[j * K + j]);", "gram[i * K + i], gram[i * K + i]);"),
     ("forced_ignored", "if (forced && forced[t] >= 0) accept = forced[t];", ""),
     ("average_not_divided", "out[d] = sum / (double)K;", "out[d] = sum;"),
+    ("bucket_offset_ignored", "sub[i] = (const char *)grads[i] + (size_t)lo * esize;", "sub[i] = (const char *)grads[i];"),
+    ("bucket_mask_row", "mask + (size_t)b * K, dist + (size_t)b * K,", "mask, dist + (size_t)b * K,"),
+    ("bucket_output_not_offset", "order, NULL, g + lo,", "order, NULL, g,"),
     ("ring_order_not_rotated", "for (int t = 0; t < K; ++t) order[t] = (s + t) % K;",
      "for (int t = 0; t < K; ++t) order[t] = t;"),
     ("ring_ties_to_last", "if (c > best_count) { best_count = c; best_seed = s; }",
