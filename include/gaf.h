@@ -45,6 +45,7 @@ extern "C" {
 #endif
 
 #define GAF_MAX_K 64            /* largest number of micro-gradients per call */
+#define GAF_MAX_BUCKETS 256     /* largest number of buckets of the bucketed variant */
 
 enum { GAF_F32 = 0, GAF_BF16 = 1 };
 
@@ -168,6 +169,28 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
                                    double tau,
                                    float *macro_out, uint8_t *mask_out, float *dist_out,
                                    int32_t *count_out, int32_t *seed_out,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Bucketed variant.  Section 5 notes that inside a ring all-reduce the cosine distance
+ * would be applied "to buckets at a time": here the D parameters are cut into S
+ * consecutive buckets (the tensors of a network, the buckets of an all-reduce) and
+ * Algorithm 1 + Eq. 5 run on every bucket independently -- its own running sum,
+ * decisions and count.  Gram-first: one pass builds a K x K Gram matrix per bucket,
+ * the decisions are walked per bucket, one pass writes every bucket's g/c.
+ *   K           1 .. 8
+ *   S, offsets  1 <= S <= GAF_MAX_BUCKETS; HOST array of S+1 ascending element offsets,
+ *               offsets[0] = 0, offsets[S] = D; every offset but the last must be a
+ *               multiple of 8 elements (else GAF_ERR_ALIGN); empty buckets are legal
+ *   macro_out   device, D floats: bucket b holds its g/c
+ *   mask_out    device, S*K bytes, row b = bucket b, by original index
+ *   dist_out    device, S*K floats or NULL;  count_out  device, S int32
+ */
+int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, int dtype,
+                                   double tau, const int32_t *order,
+                                   int S, const int64_t *offsets,
+                                   float *macro_out, uint8_t *mask_out, float *dist_out,
+                                   int32_t *count_out,
                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*

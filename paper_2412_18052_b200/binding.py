@@ -25,6 +25,7 @@ EXPORTS = [
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
     "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
     "gaf_filter_accumulate_any_seed", "gaf_stream_begin", "gaf_stream_push", "gaf_stream_end",
+    "gaf_filter_accumulate_bucketed",
 ]
 
 
@@ -59,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.gaf_last_launch_count.argtypes = []
         L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.gaf_filter_accumulate_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gaf_filter_accumulate_bucketed.argtypes = [vp, i32, i64, i32, dbl, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.gaf_stream_begin.argtypes = [vp, i64, i32, vp, vp, sz, vp]
         L.gaf_stream_push.argtypes = [vp, i32, i64, i32, dbl, vp, vp, sz, vp]
         L.gaf_stream_end.argtypes = [i32, i64, vp, vp, vp, vp, vp, sz, vp]
@@ -199,6 +201,30 @@ def gaf_filter_accumulate_any_seed(grads: Sequence[torch.Tensor], tau: float, wo
         seed_out.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()),
         "gaf_filter_accumulate_any_seed")
     return macro_out, mask_out, dist_out, count_out, seed_out
+
+
+def gaf_filter_accumulate_bucketed(grads: Sequence[torch.Tensor], tau: float, offsets: Sequence[int],
+                                   workspace: torch.Tensor, order: Optional[Sequence[int]] = None,
+                                   macro_out: Optional[torch.Tensor] = None):
+    """Bucketed variant: Algorithm 1 + Eq. 5 independently on every bucket [offsets[b], offsets[b+1]).
+    Returns (macro[D], mask[S,K], dist[S,K], count[S]) device tensors."""
+    K, D = len(grads), grads[0].numel()
+    S = len(offsets) - 1
+    dev = grads[0].device
+    if macro_out is None:
+        macro_out = torch.empty(D, dtype=torch.float32, device=dev)
+    mask_out = torch.empty(S, K, dtype=torch.uint8, device=dev)
+    dist_out = torch.empty(S, K, dtype=torch.float32, device=dev)
+    count_out = torch.empty(S, dtype=torch.int32, device=dev)
+    ptrs = _ptr_array(grads)
+    ordp = _order_array(order)
+    offs = (ctypes.c_int64 * (S + 1))(*[int(o) for o in offsets])
+    _check(lib().gaf_filter_accumulate_bucketed(
+        ctypes.cast(ptrs, ctypes.c_void_p), K, D, _dtype_code(grads[0]), float(tau),
+        ordp and ctypes.cast(ordp, ctypes.c_void_p), S, ctypes.cast(offs, ctypes.c_void_p),
+        macro_out.data_ptr(), mask_out.data_ptr(), dist_out.data_ptr(), count_out.data_ptr(),
+        workspace.data_ptr(), workspace.numel(), _stream()), "gaf_filter_accumulate_bucketed")
+    return macro_out, mask_out, dist_out, count_out
 
 
 def gaf_stream_begin(seed: torch.Tensor, acc: torch.Tensor, workspace: torch.Tensor) -> None:

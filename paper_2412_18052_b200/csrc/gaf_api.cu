@@ -6,6 +6,7 @@
 #include <cstring>
 
 #include "../../include/gaf.h"
+#include "gaf_bucketed.cuh"
 #include "gaf_device.cuh"
 #include "gaf_gram_tc.cuh"
 #include "gaf_gramfilter.cuh"
@@ -66,7 +67,14 @@ size_t gram_partials_bytes(int K) {
     return pairs * kGramMaxSlices * 64 * sizeof(double);
 }
 size_t gram_matrix_bytes(int K) { return round_up(size_t(K) * K * sizeof(double), 256); }
-size_t pairwise_extra_bytes(int K) { return gram_partials_bytes(K) + 3 * gram_matrix_bytes(K); }
+// Bucketed variant: partial slots [ctas + buckets][64] doubles and one bit mask per bucket.
+size_t bucketed_extra_bytes() {
+    return size_t(kBkMaxCtas + kBkMaxBuckets) * 64 * sizeof(double) + size_t(kBkMaxBuckets) * 8;
+}
+size_t pairwise_extra_bytes(int K) {
+    const size_t a = gram_partials_bytes(K) + 3 * gram_matrix_bytes(K), b = bucketed_extra_bytes();
+    return a > b ? a : b;
+}
 
 // Tiled Gram matrix of K gradients (by original index) into the workspace; optional
 // distance matrix.  Two launches.
@@ -249,6 +257,26 @@ int check_grads(const void *const *grads, int K, int64_t D, int dtype) {
     return GAF_OK;
 }
 
+template <typename T, int KT>
+void launch_bucket_gram_kt(const BucketGramArgs &a, const BucketTable &bt, int grid, cudaStream_t st) {
+    bucket_gram_kernel<T, KT><<<grid, kBkThreads, 0, st>>>(a, bt);
+}
+template <typename T>
+int launch_bucket_gram(const BucketGramArgs &a, const BucketTable &bt, int K, int grid, cudaStream_t st) {
+    switch (K) {
+        case 1: launch_bucket_gram_kt<T, 1>(a, bt, grid, st); break;
+        case 2: launch_bucket_gram_kt<T, 2>(a, bt, grid, st); break;
+        case 3: launch_bucket_gram_kt<T, 3>(a, bt, grid, st); break;
+        case 4: launch_bucket_gram_kt<T, 4>(a, bt, grid, st); break;
+        case 5: launch_bucket_gram_kt<T, 5>(a, bt, grid, st); break;
+        case 6: launch_bucket_gram_kt<T, 6>(a, bt, grid, st); break;
+        case 7: launch_bucket_gram_kt<T, 7>(a, bt, grid, st); break;
+        case 8: launch_bucket_gram_kt<T, 8>(a, bt, grid, st); break;
+        default: return GAF_ERR_ARG;
+    }
+    return GAF_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -404,6 +432,79 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
                                    seed_out, base, di.sms, di.l2_bytes, st)
         : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
                                            count_out, seed_out, base, di.sms, di.l2_bytes, st);
+}
+
+int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, int dtype, double tau,
+                                   const int32_t *order, int S, const int64_t *offsets, float *macro_out,
+                                   uint8_t *mask_out, float *dist_out, int32_t *count_out, void *workspace,
+                                   size_t workspace_bytes, void *cuda_stream) {
+    g_launches = 0;
+    if (int rc = check_grads(grads, K, D, dtype)) return rc;
+    if (K > kGsMaxK) return GAF_ERR_UNSUPPORTED;
+    if ((!macro_out && D > 0) || !mask_out || !count_out || !offsets || tau != tau) return GAF_ERR_ARG;
+    if (S < 1 || S > GAF_MAX_BUCKETS || offsets[0] != 0 || offsets[S] != D) return GAF_ERR_ARG;
+    for (int b = 0; b < S; ++b) {
+        if (offsets[b + 1] < offsets[b]) return GAF_ERR_ARG;
+        if (b > 0 && (offsets[b] & 7) != 0) return GAF_ERR_ALIGN;
+    }
+    if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
+    int32_t ord[GAF_MAX_K];
+    {
+        bool seen[GAF_MAX_K] = {false};
+        for (int t = 0; t < K; ++t) {
+            const int32_t i = order ? order[t] : t;
+            if (i < 0 || i >= K || seen[i]) return GAF_ERR_ARG;
+            seen[i] = true;
+            ord[t] = i;
+        }
+    }
+    {
+        const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
+        for (int i = 0; i < K; ++i) {
+            const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
+            const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
+            if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
+        }
+    }
+    if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + bucketed_extra_bytes())) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return GAF_ERR_CUDA;
+    auto *base = static_cast<unsigned char *>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    BucketTable bt{};
+    bt.S = S;
+    for (int b = 0; b <= S; ++b) bt.off[b] = offsets[b];
+    double *partials = reinterpret_cast<double *>(base + kExtraOffset);
+    unsigned long long *bits = reinterpret_cast<unsigned long long *>(
+        base + kExtraOffset + size_t(kBkMaxCtas + kBkMaxBuckets) * 64 * sizeof(double));
+    int grid = di.sms * 2;
+    if (grid > kBkMaxCtas) grid = kBkMaxCtas;
+    const int64_t n_oct = D / kOct;
+    if (n_oct < grid) grid = n_oct > 0 ? int(n_oct) : 1;
+
+    BucketGramArgs ga{};
+    for (int t = 0; t < K; ++t) ga.g[t] = grads[ord[t]];
+    ga.D = D; ga.partials = partials; ga.ctl = reinterpret_cast<Control *>(base);
+    int rc = dtype == GAF_F32 ? launch_bucket_gram<float>(ga, bt, K, grid, st)
+                              : launch_bucket_gram<__nv_bfloat16>(ga, bt, K, grid, st);
+    if (rc != GAF_OK) return rc;
+    ++g_launches;
+
+    BucketWalkArgs wa{};
+    wa.K = K; wa.D = D; wa.ctas = grid; wa.tau = tau; wa.partials = partials; wa.mask_out = mask_out;
+    wa.dist_out = dist_out; wa.count_out = count_out; wa.bits = bits; wa.ctl = ga.ctl;
+    for (int t = 0; t < K; ++t) wa.idx[t] = ord[t];
+    bucket_walk_kernel<<<S, 64 * kWalkChains, 0, st>>>(wa, bt);
+    ++g_launches;
+
+    BucketMeanArgs ma{};
+    for (int t = 0; t < K; ++t) ma.g[t] = grads[ord[t]];
+    ma.K = K; ma.D = D; ma.out = macro_out; ma.bits = bits;
+    if (dtype == GAF_F32) bucket_mean_kernel<float><<<grid, kBkThreads, 0, st>>>(ma, bt);
+    else bucket_mean_kernel<__nv_bfloat16><<<grid, kBkThreads, 0, st>>>(ma, bt);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }
 
 int gaf_stream_begin(const void *seed, int64_t D, int dtype, float *acc, void *workspace,

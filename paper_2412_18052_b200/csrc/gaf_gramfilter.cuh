@@ -244,21 +244,27 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     const int64_t n_vec = a.D / N;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int since_flush = 0;
-    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n_vec; q += stride) {
-        float x[KT][N];
-        const uint64_t pol = (q * N >= a.keep_from) ? pol_last : pol_first;
+    // The trip count is the same for all lanes of a warp (the bound is tested on the warp's first
+    // vector): the flush below shuffles across the whole warp, so the lanes must reach it together.
+    const int64_t warp_first = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31);
+    for (int64_t qw = warp_first; qw < n_vec; qw += stride) {
+        const int64_t q = qw + lane;
+        if (q < n_vec) {
+            float x[KT][N];
+            const uint64_t pol = (q * N >= a.keep_from) ? pol_last : pol_first;
 #pragma unroll
-        for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], q * N, pol, x[r]);
-        int p = 0;
+            for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], q * N, pol, x[r]);
+            int p = 0;
 #pragma unroll
-        for (int r = 0; r < KT; ++r)
+            for (int r = 0; r < KT; ++r)
 #pragma unroll
-            for (int c = r; c < KT; ++c, ++p) {
-                float s = acc[p];
+                for (int c = r; c < KT; ++c, ++p) {
+                    float s = acc[p];
 #pragma unroll
-                for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
-                acc[p] = s;
-            }
+                    for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
+                    acc[p] = s;
+                }
+        }
         if (++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
     }
     // ragged tail (D mod N elements), first CTA

@@ -93,25 +93,30 @@ __global__ void __launch_bounds__(kGramThreads) gram_tile_kernel(GramArgs a) {
     const int64_t n_quad = a.D / 4;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int since_flush = 0;
-    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n_quad; q += stride) {
-        float xi[kGramTile][4], xj[kGramTile][4];
+    // warp-uniform trip count: the flush shuffles across the whole warp
+    const int64_t warp_first = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31);
+    for (int64_t qw = warp_first; qw < n_quad; qw += stride) {
+        const int64_t q = qw + lane;
+        if (q < n_quad) {
+            float xi[kGramTile][4], xj[kGramTile][4];
 #pragma unroll
-        for (int r = 0; r < kGramTile; ++r) load4<T>(ri[r], q * 4, xi[r]);
-        if (!diag) {
+            for (int r = 0; r < kGramTile; ++r) load4<T>(ri[r], q * 4, xi[r]);
+            if (!diag) {
 #pragma unroll
-            for (int r = 0; r < kGramTile; ++r) load4<T>(rj[r], q * 4, xj[r]);
-        }
-#pragma unroll
-        for (int r = 0; r < kGramTile; ++r)
-#pragma unroll
-            for (int c = 0; c < kGramTile; ++c) {
-                if (diag && c < r) continue;
-                const float *y = diag ? xi[c] : xj[c];
-                float s = acc[r][c];
-                s = fmaf(xi[r][0], y[0], s); s = fmaf(xi[r][1], y[1], s);
-                s = fmaf(xi[r][2], y[2], s); s = fmaf(xi[r][3], y[3], s);
-                acc[r][c] = s;
+                for (int r = 0; r < kGramTile; ++r) load4<T>(rj[r], q * 4, xj[r]);
             }
+#pragma unroll
+            for (int r = 0; r < kGramTile; ++r)
+#pragma unroll
+                for (int c = 0; c < kGramTile; ++c) {
+                    if (diag && c < r) continue;
+                    const float *y = diag ? xi[c] : xj[c];
+                    float s = acc[r][c];
+                    s = fmaf(xi[r][0], y[0], s); s = fmaf(xi[r][1], y[1], s);
+                    s = fmaf(xi[r][2], y[2], s); s = fmaf(xi[r][3], y[3], s);
+                    acc[r][c] = s;
+                }
+        }
         if (++since_flush == kGramFlushEvery) { flush(); since_flush = 0; }
     }
     // ragged tail (D mod 4 elements): lanes 0..2 of warp 0 in slice 0

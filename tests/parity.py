@@ -157,3 +157,26 @@ def check_any_seed(grads: Sequence[torch.Tensor], tau: float, workspace: torch.T
     plain = gaf.gaf_filter_accumulate(grads, tau, workspace, order=order)
     assert torch.equal(plain[0], macro) and torch.equal(plain[1], mask)
     return {"seed": g_seed, "count": r.count, "counts": counts.tolist()}
+
+
+def check_bucketed(grads: Sequence[torch.Tensor], tau: float, offsets, workspace: torch.Tensor,
+                   order: Optional[Sequence[int]] = None):
+    """gaf_filter_accumulate_bucketed against the oracle, bucket by bucket (with the
+    near-tau replay rule applied per bucket)."""
+    K, D = len(grads), grads[0].numel()
+    S = len(offsets) - 1
+    macro, mask, dist, count = gaf.gaf_filter_accumulate_bucketed(grads, tau, offsets, workspace, order=order)
+    np_grads = [as_numpy_bits(g) for g in grads]
+    g_macro = macro.cpu().numpy()
+    g_mask, g_dist, g_count = mask.cpu().numpy(), dist.cpu().numpy().astype(np.float64), count.cpu().numpy()
+    patterns = set()
+    for b in range(S):
+        lo, hi = offsets[b], offsets[b + 1]
+        sub = [g[lo:hi] for g in np_grads]
+        r, _ = oracle_with_replay(sub, tau, order, g_mask[b])
+        assert g_mask[b].tolist() == r.mask.tolist() and int(g_count[b]) == r.count, (b, lo, hi)
+        assert float(np.max(np.abs(g_dist[b] - r.dist))) <= DIST_ATOL, (b, g_dist[b], r.dist)
+        if hi > lo:
+            assert rel_l2(g_macro[lo:hi], r.out) <= MACRO_RTOL[grads[0].dtype], (b, lo, hi)
+        patterns.add(tuple(g_mask[b].tolist()))
+    return patterns

@@ -8,7 +8,7 @@ import torch
 
 import paper_2412_18052_b200 as gaf
 from paper_2412_18052_b200 import workloads
-from parity import check_any_seed, check_cosdist, check_filter, check_pairwise
+from parity import check_any_seed, check_bucketed, check_cosdist, check_filter, check_pairwise
 
 pytestmark = pytest.mark.gpu
 
@@ -216,6 +216,20 @@ def test_filter_random_cases(ws):
         check_filter(w.grads, tau, ws, order=order, schedule=schedule, expect_status=None)
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_gram_loop_ends_inside_a_warp_at_the_flush_period(ws, dtype):
+    """Lengths for which some lanes of a warp run exactly 16 rounds of the Gram loop (one
+    binary64 flush, a warp-wide shuffle) and their neighbours 15: the flush must still be
+    reached by whole warps."""
+    threads = 2 * torch.cuda.get_device_properties(0).multi_processor_count * 512
+    per_vec = 4 if dtype == "f32" else 8
+    for extra in (1000, 40):
+        D = (threads * 15 + extra) * per_vec + 3
+        w = _mix(3, D, dtype, seed=77, rho=[0.7, 0.5, -0.4])
+        check_filter(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_GRAM)
+        check_pairwise(w.grads, ws)
+
+
 def test_filter_partly_cancelling_gradients(ws):
     """Accepted gradients that nearly cancel: the norm of the running sum is a small
     difference of large Gram entries in the Gram-first schedule."""
@@ -271,6 +285,56 @@ def test_any_seed_variant(ws, dtype):
         w = _mix(K, Dk, dtype, seed=900 + K)
         r = check_any_seed(w.grads, 0.97, ws)
         assert r["count"] == max(r["counts"])
+
+
+# ------------------------------------------------------------ bucketed variant --
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_bucketed_variant(ws, dtype):
+    # one bucket = the plain filter
+    w = _mix(4, 100_003, dtype, seed=31, rho=[0.8, 0.6, -0.2, 0.7])
+    check_bucketed(w.grads, 0.8, [0, w.D], ws)
+    plain = gaf.gaf_filter_accumulate(w.grads, 0.8, ws)
+    buck = gaf.gaf_filter_accumulate_bucketed(w.grads, 0.8, [0, w.D], ws)
+    assert torch.equal(plain[0], buck[0]) and torch.equal(plain[1], buck[1][0])
+    # many buckets of very different sizes, empty ones, a ragged end, a non-identity order
+    rng = np.random.RandomState(7)
+    for K, D in ((1, 5000), (2, 64), (3, 300_011), (5, 2_000_005), (8, 777_777)):
+        cuts = sorted(set(int(x) // 8 * 8 for x in rng.randint(0, D, size=24)) | {0})
+        offsets = cuts + [cuts[-1], D] if cuts[-1] < D else cuts + [D]
+        offsets = [0] + [o for o in offsets[1:]]
+        if offsets[1] != 0:
+            offsets.insert(1, 0)                                    # an empty first bucket
+        w = _mix(K, D, dtype, seed=400 + K)
+        for g in w.grads[1:2]:
+            g[: D // 3] = -w.grads[0][: D // 3]                       # buckets must disagree with each other
+        order = [int(x) for x in rng.permutation(K)]
+        patterns = check_bucketed(w.grads, 0.9, offsets, ws, order=order)
+        if K >= 3:
+            assert len(patterns) >= 2
+
+
+def test_bucketed_resnet18_layout(ws):
+    """Configuration 2 cut at its 62 parameter tensors."""
+    w = workloads.config(2, device="cuda")
+    sizes = workloads.resnet18_tensor_sizes(100)
+    offsets = [0] + list(np.cumsum(sizes))
+    assert offsets[-1] == w.D and len(offsets) == 63
+    check_bucketed(w.grads, 0.97, [int(o) for o in offsets], ws)
+
+
+def test_bucketed_argument_errors(ws):
+    w = _mix(3, 1000, "f32", seed=1)
+    for bad in ([0, 500], [1, 1000], [0, 700, 600, 1000]):
+        with pytest.raises(gaf.GafError) as e:
+            gaf.gaf_filter_accumulate_bucketed(w.grads, 0.9, bad, ws)
+        assert e.value.code == 1
+    with pytest.raises(gaf.GafError) as e:
+        gaf.gaf_filter_accumulate_bucketed(w.grads, 0.9, [0, 100, 1000], ws)      # 100 is not a multiple of 8
+    assert e.value.code == 2
+    with pytest.raises(gaf.GafError) as e:
+        gaf.gaf_filter_accumulate_bucketed(_mix(9, 1000, "f32", seed=2).grads, 0.9, [0, 1000], ws)
+    assert e.value.code == 7
 
 
 # ------------------------------------------------- the named configurations --
