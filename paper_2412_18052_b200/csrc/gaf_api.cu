@@ -8,6 +8,7 @@
 #include "../../include/gaf.h"
 #include "gaf_bucketed.cuh"
 #include "gaf_device.cuh"
+#include "gaf_fused.cuh"
 #include "gaf_gram_tc.cuh"
 #include "gaf_gramfilter.cuh"
 #include "gaf_pairwise.cuh"
@@ -23,6 +24,9 @@ thread_local int g_launches = 0;
 struct DeviceInfo {
     int sms = 0;
     int l2_bytes = 0;
+    int smem_per_sm = 0;                // shared memory of one SM
+    int smem_per_cta_max = 0;           // opt-in limit of one CTA
+    int cooperative = 0;                // cooperative launches supported
 };
 
 // Attributes of the current device (queried per call: a cheap driver lookup).
@@ -31,6 +35,11 @@ bool device_info(DeviceInfo *out) {
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&out->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&out->l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&out->smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
+        return false;
+    if (cudaDeviceGetAttribute(&out->smem_per_cta_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+        return false;
+    if (cudaDeviceGetAttribute(&out->cooperative, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return false;
     return out->sms > 0;
 }
 
@@ -158,12 +167,85 @@ int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
     }
 }
 
+// One-launch form of the Gram-first schedule (gaf_fused.cuh).  Returns GAF_OK when it was
+// launched, -1 when this device or size does not allow it (the caller then takes the two-launch
+// form), or an error code.
+int g_carveout_pct = -1;
+int g_keep_l2_pct = 10;                 // share of L2 the Gram pass asks to keep for the second pass
+int g_park_rounds_max = 2;
+constexpr int64_t kFusedMaxInputBytes = int64_t(1) << 30;   // beyond this nothing stays on chip anyway
+
+template <typename T, int KT>
+int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st) {
+    auto kernel = gram_fused_kernel<T, KT>;
+    // CTAs per SM by registers alone, then as many parked rounds as shared memory allows
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kGsThreads, 0) != cudaSuccess || occ < 1)
+        return -1;
+    if (occ > 2) occ = 2;
+    cudaFuncAttributes fa{};
+    if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return GAF_ERR_CUDA;
+    const int round_bytes = KT * kGsThreads * 16;
+    int64_t budget = di.smem_per_sm / occ - 1024 - int64_t(fa.sharedSizeBytes);
+    if (budget > di.smem_per_cta_max - int64_t(fa.sharedSizeBytes)) budget = di.smem_per_cta_max - int64_t(fa.sharedSizeBytes);
+    int park = budget > 0 ? int(budget / round_bytes) : 0;
+    if (park > g_park_rounds_max) park = g_park_rounds_max;
+    const int dyn = park * round_bytes;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+        return GAF_ERR_CUDA;
+    {
+        // shared memory share of the L1/shared array: what the CTAs of one SM need, no more (the rest is L1)
+        int pct = g_carveout_pct >= 0 ? g_carveout_pct
+                                      : int((int64_t(dyn + fa.sharedSizeBytes + 1024) * occ * 100 + di.smem_per_sm - 1) / di.smem_per_sm);
+        if (pct > 100) pct = 100;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, pct) != cudaSuccess)
+            return GAF_ERR_CUDA;
+    }
+    int occ2 = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ2, kernel, kGsThreads, dyn) != cudaSuccess || occ2 < 1)
+        return -1;
+    if (occ2 < occ) occ = occ2;
+    int64_t grid = int64_t(di.sms) * occ;
+    if (grid > kGsMaxCtas) grid = kGsMaxCtas;
+    const int64_t work = (a.D / FusedVec<T>::N + kGsThreads - 1) / kGsThreads;
+    if (grid > work) grid = work;
+    if (grid < 1) grid = 1;
+    a.park_rounds = park;
+    // the last stretch is asked to stay in L2 for the second pass
+    const int64_t per_elem = int64_t(KT) * int64_t(sizeof(T));
+    const int64_t keep_elems = int64_t(di.l2_bytes) * g_keep_l2_pct / 100 / per_elem;
+    a.keep_from = a.D > keep_elems ? a.D - keep_elems : 0;
+    void *params[] = {&a};
+    const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kernel), dim3(int(grid)),
+                                                        dim3(kGsThreads), params, size_t(dyn), st);
+    if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+    ++g_launches;
+    return GAF_OK;
+}
+
+template <typename T>
+int launch_gram_fused(GramFusedArgs &a, int K, const DeviceInfo &di, cudaStream_t st) {
+    if (!di.cooperative || g_park_rounds_max < 0) return -1;
+    if (int64_t(K) * int64_t(sizeof(T)) * a.D > kFusedMaxInputBytes) return -1;
+    switch (K) {
+        case 2: return launch_gram_fused_kt<T, 2>(a, di, st);
+        case 3: return launch_gram_fused_kt<T, 3>(a, di, st);
+        case 4: return launch_gram_fused_kt<T, 4>(a, di, st);
+        case 5: return launch_gram_fused_kt<T, 5>(a, di, st);
+        case 6: return launch_gram_fused_kt<T, 6>(a, di, st);
+        case 7: return launch_gram_fused_kt<T, 7>(a, di, st);
+        case 8: return launch_gram_fused_kt<T, 8>(a, di, st);
+        default: return -1;
+    }
+}
+
 // Gram-first schedule: Gram matrix, scalar walk of Algorithm 1, masked mean.
 // `seed_out` non-null selects the any-seed variant (ord must then be the identity).
 template <typename T>
 int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double tau, const int32_t *ord,
                       float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
-                      int32_t *seed_out, unsigned char *base, int sms, int l2_bytes, cudaStream_t st) {
+                      int32_t *seed_out, unsigned char *base, const DeviceInfo &di, cudaStream_t st) {
+    const int sms = di.sms;
     Control *ctl = reinterpret_cast<Control *>(base);
     RingArgs ring{};
     if (seed_out) {
@@ -177,12 +259,23 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     double *gram_by_step = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K) +
                                                       gram_matrix_bytes(K));
     if (use_small_gram(K, D, dtype)) {
+        // short calls: both passes in one co-resident launch
+        GramFusedArgs f{};
+        for (int t = 0; t < K; ++t) f.g[t] = g[ord[t]];
+        f.D = D; f.out = macro_out;
+        f.partials = reinterpret_cast<double *>(base + kExtraOffset);
+        f.gram = gram_by_step;
+        f.replay = r;
+        f.ring = ring;
+        const int frc = launch_gram_fused<T>(f, K, di, st);
+        if (frc >= 0) return frc;
+
         GramSmallArgs a{};
         for (int t = 0; t < K; ++t) a.g[t] = g[ord[t]];
         a.D = D;
         // how much of the tail of the Gram pass should stay in L2 for the masked-mean pass
         const int64_t per_elem = int64_t(K) * int64_t(sizeof(T));
-        const int64_t keep_elems = int64_t(l2_bytes) * 6 / 10 / per_elem;
+        const int64_t keep_elems = int64_t(di.l2_bytes) * g_keep_l2_pct / 100 / per_elem;
         a.keep_from = D > keep_elems ? D - keep_elems : 0;
         a.partials = reinterpret_cast<double *>(base + kExtraOffset);
         a.gram = gram_by_step;
@@ -380,9 +473,9 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
             return rc;
         return dtype == GAF_F32
             ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                       count_out, nullptr, base, di.sms, di.l2_bytes, st)
+                                       count_out, nullptr, base, di, st)
             : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                               count_out, nullptr, base, di.sms, di.l2_bytes, st);
+                                               count_out, nullptr, base, di, st);
     }
     return dtype == GAF_F32
         ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
@@ -429,9 +522,9 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
     }
     return dtype == GAF_F32
         ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out, count_out,
-                                   seed_out, base, di.sms, di.l2_bytes, st)
+                                   seed_out, base, di, st)
         : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                           count_out, seed_out, base, di.sms, di.l2_bytes, st);
+                                           count_out, seed_out, base, di, st);
 }
 
 int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, int dtype, double tau,

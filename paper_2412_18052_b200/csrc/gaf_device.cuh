@@ -27,6 +27,10 @@ struct Control {
     double sums[GAF_MAX_K][3];          // by step t: {g_i.g, |g|^2, |g_i|^2}
     float stream_dist[GAF_MAX_K];       // streaming form: distance of arrival t
     uint8_t stream_mask[GAF_MAX_K];     // streaming form: decision of arrival t
+    // One-launch Gram-first schedule: the word the waiting CTAs poll, alone in its cache line.
+    // Bits 16..31 call generation, 8..15 winning seed + 1 (0: no any-seed walk), 0..7 accept bits.
+    alignas(128) unsigned int fused_word;
+    unsigned int fused_pad[31];
 };
 constexpr size_t kControlBytes = 4096;  // sizeof(Control) rounded up
 static_assert(sizeof(Control) <= kControlBytes, "control block");

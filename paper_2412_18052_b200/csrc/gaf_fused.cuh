@@ -1,0 +1,296 @@
+// Gram-first schedule of Algorithm 1 as ONE persistent launch (K <= 8).
+//
+// The two-launch form (gaf_gramfilter.cuh) reads every gradient once for the Gram
+// matrix and the accepted ones a second time for g/c (Eq. 5).  When the whole call
+// lasts tens of microseconds, what the second pass has to fetch again is a large part
+// of the cost.  Here one co-resident grid does both passes, so that what a thread
+// loaded last in the first pass is still ON CHIP when the second pass starts:
+//   pass 1   every thread walks its vectors (grid-stride), accumulating the Gram
+//            partial sums exactly as gram_small_kernel does, and parks the raw loads
+//            of its last R rounds in shared memory;
+//   decide   per-CTA partials, last CTA to arrive totals them in fixed order, walks
+//            Algorithm 1 (Eq. 4 in binary64) on the Gram matrix and publishes the accept
+//            bits; the other CTAs wait for it (bounded spin on a generation word);
+//   pass 2   the same thread visits the same vectors: the parked rounds straight from
+//            shared memory, then the rest from the end towards the start (the rounds
+//            just before the parked ones were loaded "keep in L2"), adding the accepted
+//            gradients in processing order in binary32 and dividing by c.
+// Same sums, same order of additions as the two-launch form: identical outputs.
+// The grid must be co-resident (cooperative launch); every wait is bounded and ends in
+// GAF_STATUS_TIMEOUT.
+#pragma once
+
+#include "gaf_device.cuh"
+#include "gaf_gramfilter.cuh"
+
+namespace gaf {
+
+constexpr unsigned int kFusedSpinLimit = 1u << 22;   // polls of >= 200 ns each: about a second
+
+struct GramFusedArgs {
+    const void *g[kGsMaxK];                 // processing order (original order in any-seed mode)
+    int64_t D;
+    int64_t keep_from;                      // elements from here on are loaded "keep in L2"
+    int park_rounds;                        // R: rounds per thread parked in shared memory
+    double *partials;                       // [pair][kGsPartialStride]
+    double *gram;                           // [K][K]
+    float *out;                             // D floats
+    ReplayArgs replay;                      // used when ring.K == 0
+    RingArgs ring;                          // any-seed mode when ring.K > 0
+};
+
+// The polled word carries its own payload, so no ordering with other memory is needed.
+__device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int *p) {
+    unsigned int v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u32(unsigned int *p, unsigned int v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+template <typename T> struct FusedVec;      // one 16-byte vector of a gradient, widened
+template <> struct FusedVec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void widen(const uint4 &r, float (&v)[4]) {
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y);
+        v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    }
+};
+template <> struct FusedVec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void widen(const uint4 &r, float (&v)[8]) {
+        const unsigned int w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[2 * k] = bf16_bits_to_float(w[k] & 0xFFFFu);
+            v[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+        }
+    }
+};
+
+template <int N>
+__device__ __forceinline__ void store_vec_streaming(float *dst, const float (&v)[N]) {
+#pragma unroll
+    for (int h = 0; h < N / 4; ++h)
+        __stcs(reinterpret_cast<float4 *>(dst) + h, make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]));
+}
+
+template <typename T, int KT>
+__global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1))
+gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
+    constexpr int NP = KT * (KT + 1) / 2;
+    constexpr int N = FusedVec<T>::N;
+    extern __shared__ uint4 parked[];       // [round][gradient][thread]
+    __shared__ double sacc[kGsThreads / 32][NP];
+    __shared__ double sgram[KT * KT];
+    __shared__ bool is_last;
+    __shared__ const T *list[kGsMaxK];      // accepted gradients in the order they are added
+    __shared__ int list_row[kGsMaxK];       // ... and their row in `parked`
+    __shared__ int n_list;                  // c, or -1 when the wait ran out
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    Control *ctl = a.replay.ctl;
+
+    // generation of the decision word before anybody can have published this call's
+    unsigned int gen0 = 0, decided = 0;
+    if (tid == 0) {
+        gen0 = ld_relaxed_u32(&ctl->fused_word) >> 16;
+        if (blockIdx.x == 0) ctl->status = 0;
+    }
+    for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
+    __syncwarp();
+
+    const T *row[KT];
+#pragma unroll
+    for (int r = 0; r < KT; ++r) row[r] = static_cast<const T *>(a.g[r]);
+
+    const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
+    const int64_t n_vec = a.D / N;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    // rounds of this warp (the same for all its lanes: the flush shuffles across the warp)
+    const int64_t warp_first = (int64_t)blockIdx.x * blockDim.x + (tid & ~31);
+    const int64_t rounds = warp_first < n_vec ? (n_vec - warp_first + stride - 1) / stride : 0;
+    const int64_t parked_rounds = rounds < a.park_rounds ? rounds : a.park_rounds;   // the FIRST ones
+    float acc[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) acc[p] = 0.0f;
+    auto flush = [&]() {
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            float v = acc[p];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
+            if (lane == 0) sacc[warp][p] += (double)v;
+            acc[p] = 0.0f;
+        }
+    };
+
+    const int64_t tail0 = n_vec * N;
+    // ---- pass 1: Gram partial sums; the last rounds stay in shared memory ----
+    int since_flush = 0;
+    for (int64_t j = 0; j < rounds; ++j) {
+        const int64_t q = warp_first + j * stride + lane;
+        if (q < n_vec) {
+            const bool park = j < parked_rounds;
+            const uint64_t pol = (q * N >= a.keep_from) ? pol_last : pol_first;
+            uint4 raw[KT];
+#pragma unroll
+            for (int r = 0; r < KT; ++r) raw[r] = ld16_policy(row[r] + q * N, pol);
+            if (park) {
+                uint4 *slot = parked + (size_t)j * KT * kGsThreads + tid;
+#pragma unroll
+                for (int r = 0; r < KT; ++r) slot[r * kGsThreads] = raw[r];
+            }
+            float x[KT][N];
+#pragma unroll
+            for (int r = 0; r < KT; ++r) FusedVec<T>::widen(raw[r], x[r]);
+            int p = 0;
+#pragma unroll
+            for (int r = 0; r < KT; ++r)
+#pragma unroll
+                for (int c = r; c < KT; ++c, ++p) {
+                    float s = acc[p];
+#pragma unroll
+                    for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
+                    acc[p] = s;
+                }
+        }
+        if (++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+    }
+    // ragged tail (D mod N elements), first CTA
+    if (blockIdx.x == 0 && tail0 + tid < a.D) {
+        const int64_t e = tail0 + tid;
+        float x[KT];
+#pragma unroll
+        for (int r = 0; r < KT; ++r) x[r] = load1<T>(row[r], e);
+        int p = 0;
+#pragma unroll
+        for (int r = 0; r < KT; ++r)
+#pragma unroll
+            for (int c = r; c < KT; ++c, ++p) acc[p] = fmaf(x[r], x[c], acc[p]);
+    }
+    flush();
+    __syncthreads();
+    if (tid < NP) {
+        double s = 0.0;
+        for (int w = 0; w < kGsThreads / 32; ++w) s += sacc[w][tid];
+        a.partials[(size_t)tid * kGsPartialStride + blockIdx.x] = s;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int old = atomicInc(&ctl->ticket, gridDim.x - 1);
+        is_last = (old == gridDim.x - 1);
+    }
+    __syncthreads();
+
+    // ---- decide: last CTA totals the partials in fixed order and walks Algorithm 1 ----
+    if (is_last) {
+        __threadfence();
+        total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
+        __syncthreads();
+        // the accept bits go out first, in the polled word itself; the outputs follow
+        auto notice = [&](int seed, unsigned long long bits) {
+            const unsigned int word = ((gen0 + 1u) << 16) | ((unsigned int)(seed + 1) << 8) | (unsigned int)(bits & 0xFFull);
+            decided = word;
+            st_relaxed_u32(&ctl->fused_word, word);
+        };
+        if (a.ring.K > 0) {
+            __shared__ int ring_count[kGsMaxK];
+            __shared__ unsigned long long ring_bits[kGsMaxK];
+            ring_replay_on_gram(a.ring, sgram, ring_count, ring_bits, notice);
+        } else {
+            __shared__ ReplayTable table;
+            replay_on_gram_parallel(a.replay, sgram, table, [&](unsigned long long bits) { notice(-1, bits); });
+        }
+    }
+    if (tid == 0) {
+        unsigned int word = decided;
+        bool ok = true;
+        if (!is_last) {
+            unsigned int polls = 0;
+            while (((word = ld_relaxed_u32(&ctl->fused_word)) >> 16) == gen0) {
+                __nanosleep(200);
+                if (++polls > kFusedSpinLimit) { ok = false; break; }
+            }
+        }
+        if (!ok) {
+            atomicOr(&ctl->status, GAF_STATUS_TIMEOUT);
+            n_list = -1;
+        } else {
+            const unsigned int bits = word & 0xFFu;
+            const int seed = (int)((word >> 8) & 0xFFu) - 1;
+            const int start = seed < 0 ? 0 : seed;
+            int n = 0;
+            for (int t = 0; t < KT; ++t) {
+                const int i = (start + t) % KT;
+                if ((bits >> i) & 1u) { list[n] = static_cast<const T *>(a.g[i]); list_row[n] = i; ++n; }
+            }
+            n_list = n;
+        }
+    }
+    __syncthreads();
+    const int n = n_list;
+    if (n < 0) return;
+    const float cdiv = (float)n;
+
+    // ---- pass 2a: the rounds that were not parked, last first (the most recently read lines
+    //      are the ones still in L2), two rounds in flight per thread ----
+    constexpr int U = 2;
+    for (int64_t j0 = rounds - 1; j0 >= parked_rounds; j0 -= U) {
+        int64_t q[U];
+        bool ok[U];
+        uint4 w[U][KT];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            q[u] = warp_first + (j0 - u) * stride + lane;
+            ok[u] = (j0 - u) >= parked_rounds && q[u] < n_vec;
+#pragma unroll
+            for (int i = 0; i < KT; ++i)
+                if (ok[u] && i < n) w[u][i] = ld16_policy(list[i] + q[u] * N, pol_first);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (ok[u]) {
+                float v[N];
+                FusedVec<T>::widen(w[u][0], v);
+#pragma unroll
+                for (int i = 1; i < KT; ++i)
+                    if (i < n) {
+                        float x[N];
+                        FusedVec<T>::widen(w[u][i], x);
+#pragma unroll
+                        for (int k = 0; k < N; ++k) v[k] += x[k];
+                    }
+#pragma unroll
+                for (int k = 0; k < N; ++k) v[k] = v[k] / cdiv;
+                store_vec_streaming<N>(a.out + q[u] * N, v);
+            }
+    }
+    // ---- pass 2b: the parked rounds, from shared memory ----
+    for (int64_t j = 0; j < parked_rounds; ++j) {
+        const int64_t q = warp_first + j * stride + lane;
+        if (q < n_vec) {
+            const uint4 *slot = parked + (size_t)j * KT * kGsThreads + tid;
+            float v[N];
+            FusedVec<T>::widen(slot[list_row[0] * kGsThreads], v);
+            for (int i = 1; i < n; ++i) {
+                float x[N];
+                FusedVec<T>::widen(slot[list_row[i] * kGsThreads], x);
+#pragma unroll
+                for (int k = 0; k < N; ++k) v[k] += x[k];
+            }
+#pragma unroll
+            for (int k = 0; k < N; ++k) v[k] = v[k] / cdiv;
+            store_vec_streaming<N>(a.out + q * N, v);
+        }
+    }
+    if (blockIdx.x == 0 && tail0 + tid < a.D) {
+        const int64_t e = tail0 + tid;
+        float v = load1<T>(list[0], e);
+        for (int i = 1; i < n; ++i) v += load1<T>(list[i], e);
+        a.out[e] = v / cdiv;
+    }
+}
+
+}  // namespace gaf

@@ -21,8 +21,10 @@ namespace gaf {
 constexpr int kGsThreads = 512;
 constexpr int kGsMaxK = 8;                  // gradients the one-pass register-tiled Gram handles
 constexpr int kGsMaxCtas = 296;
+constexpr int kGsPartialStride = 320;       // per-CTA partials are stored [pair][CTA]: the totalling loads coalesce
 constexpr int kGsFlushEvery = 16;           // iterations between binary64 flushes
 constexpr int kMsThreads = 512;
+constexpr int kReplayMaxK = 8;               // the table form of the walk: 2^(K-1) - 1 cases
 
 struct ReplayArgs {
     int K;
@@ -78,6 +80,79 @@ __device__ __forceinline__ unsigned long long replay_on_gram(const ReplayArgs &r
     return bits;
 }
 
+// The same walk for K <= 8 with its latency taken out of the serial part.  Step t's test depends on
+// the earlier decisions only through WHICH gradients were accepted, so one thread per (step t,
+// accept pattern of steps 1..t-1) evaluates Eq. 4 for that case -- 2^(K-1) - 1 threads, all at once --
+// and thread 0 then only follows the decisions through the table.  Every case repeats the sums of
+// the sequential walk in the same order, so the results are the same to the last bit.
+// All threads of the block call (blockDim.x >= 128).  `early(bits)` is called by thread 0 as soon as
+// the accept bits are known, before the outputs are written.
+struct ReplayTable {
+    double d[127], p[127], na[127];
+    unsigned char accept[127], status[127];
+};
+struct NoEarlyBits {
+    __device__ __forceinline__ void operator()(unsigned long long) const {}
+};
+template <typename Early = NoEarlyBits>
+__device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, const double *gram, ReplayTable &tb,
+                                                        Early early = Early()) {
+    const int K = r.K, tid = threadIdx.x;
+    const int cases = (1 << (K - 1)) - 1;
+    if (tid < cases) {
+        const int t = 32 - __clz(tid + 1);                      // tid + 1 in [2^(t-1), 2^t)
+        const unsigned int m = (unsigned int)(tid + 1) - (1u << (t - 1));
+        auto in = [&](int v) { return v == 0 || ((m >> (v - 1)) & 1u); };   // step v accepted in this case
+        double na = gram[0];
+        for (int u = 1; u < t; ++u)
+            if (in(u)) {
+                double pu = 0.0;
+                for (int v = 0; v < u; ++v)
+                    if (in(v)) pu += gram[v * K + u];
+                na = na + 2.0 * pu + gram[u * K + u];
+            }
+        double p = 0.0;
+        for (int v = 0; v < t; ++v)
+            if (in(v)) p += gram[v * K + t];
+        int status = 0;
+        const double d = cosine_distance(p, na, gram[t * K + t], &status);
+        tb.d[tid] = d; tb.p[tid] = p; tb.na[tid] = na;
+        tb.accept[tid] = (d <= r.tau) ? 1 : 0;
+        tb.status[tid] = (unsigned char)status;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned int m = 0;
+        int node[kReplayMaxK];
+        for (int t = 1; t < K; ++t) {
+            node[t] = (1 << (t - 1)) - 1 + (int)m;
+            if (tb.accept[node[t]]) m |= 1u << (t - 1);
+        }
+        const unsigned long long bits = 1ull | ((unsigned long long)m << 1);
+        early(bits);
+        Control *c = r.ctl;
+        int status = 0, count = 1;
+        c->decision[0] = 1;
+        r.mask_out[r.idx[0]] = 1;
+        if (r.dist_out) r.dist_out[r.idx[0]] = 0.0f;
+        for (int t = 1; t < K; ++t) {
+            const int i = node[t], accept = tb.accept[i];
+            c->decision[t] = accept;
+            c->sums[t][0] = tb.p[i]; c->sums[t][1] = tb.na[i]; c->sums[t][2] = gram[t * K + t];
+            r.mask_out[r.idx[t]] = (uint8_t)accept;
+            if (r.dist_out) r.dist_out[r.idx[t]] = (float)tb.d[i];
+            status |= tb.status[i];
+            count += accept;
+        }
+        c->accept_bits = bits;
+        c->ring_seed = -1;
+        c->count = count;
+        c->status = status;
+        *r.count_out = count;
+        __threadfence();
+    }
+}
+
 // Order-indifferent variant (end of Section 3.1): Algorithm 1 from every seed s with the
 // others following in ring order s, s+1, ..., K-1, 0, ..., s-1; the seed with the largest
 // accepted count wins, ties to the smallest s.  Threads 0..K-1 of the calling block each walk
@@ -120,8 +195,15 @@ __device__ __forceinline__ void ring_walk_one_seed(const RingArgs &r, const vola
     count_out = count; bits_out = bits; status_out = status;
 }
 
+// `early`, when given, is called by thread 0 with (winning seed, its accept bits) as soon as they are
+// known, before the outputs are written.
+struct NoEarlyNotice {
+    __device__ __forceinline__ void operator()(int, unsigned long long) const {}
+};
+template <typename Early = NoEarlyNotice>
 __device__ __forceinline__ void ring_replay_on_gram(const RingArgs &r, const volatile double *gram,
-                                                    int *sh_count, unsigned long long *sh_bits) {
+                                                    int *sh_count, unsigned long long *sh_bits,
+                                                    Early early = Early()) {
     const int K = r.K;
     if ((int)threadIdx.x < K) {
         int c, st;
@@ -135,6 +217,7 @@ __device__ __forceinline__ void ring_replay_on_gram(const RingArgs &r, const vol
         int best = 0;
         for (int s = 1; s < K; ++s)
             if (sh_count[s] > sh_count[best]) best = s;
+        early(best, sh_bits[best]);
         // walk the winner once more to write its distances and status
         int c, st;
         unsigned long long b;
@@ -157,7 +240,7 @@ struct GramSmallArgs {
     const void *g[kGsMaxK];                 // processing order
     int64_t D;
     int64_t keep_from;                      // elements from here on are loaded "keep in L2"
-    double *partials;                       // [cta][64]
+    double *partials;                       // [pair][kGsPartialStride]
     double *gram;                           // [K][K]
     ReplayArgs replay;                      // used when pair_dist_out is null and ring.K == 0
     float *pair_dist_out;                   // pairwise mode: K x K distances instead of the walk
@@ -206,6 +289,49 @@ template <> struct GsVec<__nv_bfloat16> {
         }
     }
 };
+
+// Fixed-order totals of the per-CTA partial sums ([pair][CTA] layout), by the whole calling block:
+// one warp per pair (several pairs per warp when there are more pairs than warps, all loads issued
+// before the first add: this is the serial tail of the call), lane-strided sums, then a shuffle tree.
+// Fills the symmetric K x K matrix in shared memory and, when `gram_out` is given, in global memory.
+template <int KT>
+__device__ __forceinline__ void total_gram_partials(const double *part, int n_ctas, double *sgram, double *gram_out) {
+    constexpr int NP = KT * (KT + 1) / 2;
+    constexpr int kWarps = kGsThreads / 32;
+    constexpr int PW = (NP + kWarps - 1) / kWarps;             // pairs per warp
+    constexpr int kRounds = (kGsMaxCtas + 31) / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double v[PW][kRounds];
+#pragma unroll
+    for (int w = 0; w < PW; ++w) {
+        const int p = warp + w * kWarps;
+#pragma unroll
+        for (int k = 0; k < kRounds; ++k) {
+            const int i = lane + 32 * k;
+            v[w][k] = (p < NP && i < n_ctas) ? __ldcg(part + (size_t)p * kGsPartialStride + i) : 0.0;
+        }
+    }
+#pragma unroll
+    for (int w = 0; w < PW; ++w) {
+        const int p = warp + w * kWarps;
+        double s = 0.0;
+#pragma unroll
+        for (int k = 0; k < kRounds; ++k) s += v[w][k];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) s += shfl_down_f64(s, d);
+        if (lane == 0 && p < NP) {
+            int r = 0, rem = p;                                 // decode p -> (r, c), r <= c
+            while (rem >= KT - r) { rem -= KT - r; ++r; }
+            const int c = r + rem;
+            sgram[r * KT + c] = s;
+            sgram[c * KT + r] = s;
+            if (gram_out) {
+                gram_out[r * KT + c] = s;
+                gram_out[c * KT + r] = s;
+            }
+        }
+    }
+}
 
 template <typename T, int KT>
 __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_constant__ GramSmallArgs a) {
@@ -289,7 +415,7 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     if (threadIdx.x < NP) {
         double s = 0.0;
         for (int w = 0; w < kGsThreads / 32; ++w) s += sacc[w][threadIdx.x];
-        a.partials[(size_t)blockIdx.x * 64 + threadIdx.x] = s;
+        a.partials[(size_t)threadIdx.x * kGsPartialStride + blockIdx.x] = s;
     }
     __threadfence();
     __syncthreads();
@@ -304,31 +430,7 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     // last CTA: fixed-order totals (one warp per pair; all of a lane's loads are issued together,
     // this is the serial tail of the call), then the scalar walk out of shared memory
     __shared__ double sgram[KT * KT];
-    const double *part = a.partials;
-    constexpr int kRounds = (kGsMaxCtas + 31) / 32;
-    for (int p = warp; p < NP; p += kGsThreads / 32) {
-        double v[kRounds];
-#pragma unroll
-        for (int k = 0; k < kRounds; ++k) {
-            const int i = lane + 32 * k;
-            v[k] = i < (int)gridDim.x ? __ldcg(part + (size_t)i * 64 + p) : 0.0;
-        }
-        double s = 0.0;
-#pragma unroll
-        for (int k = 0; k < kRounds; ++k) s += v[k];
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) s += shfl_down_f64(s, d);
-        if (lane == 0) {
-            // decode p -> (r, c), r <= c
-            int r = 0, rem = p;
-            while (rem >= KT - r) { rem -= KT - r; ++r; }
-            const int c = r + rem;
-            sgram[r * KT + c] = s;
-            sgram[c * KT + r] = s;
-            a.gram[r * KT + c] = s;
-            a.gram[c * KT + r] = s;
-        }
-    }
+    total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
     __syncthreads();
     if (a.ring.K > 0) {
         __shared__ int ring_count[kGsMaxK];
@@ -337,7 +439,8 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
         return;
     }
     if (a.pair_dist_out == nullptr) {
-        if (threadIdx.x == 0) { replay_on_gram(a.replay, sgram, true); __threadfence(); }
+        __shared__ ReplayTable table;
+        replay_on_gram_parallel(a.replay, sgram, table);
         return;
     }
     // pairwise mode: Eq. 4 for every pair
