@@ -34,6 +34,7 @@ sys.path.insert(0, ROOT)
 METRIC = "gaf_filter_accumulate micro-gradient GB/s"
 UNIT = "GB/s"
 N_SETS = 4                       # rotating input sets: each step's inputs are cold in L2
+SCHED_NAMES = {0: "auto", 1: "stepwise", 2: "gram-first, two launches", 3: "gram-first, one launch"}
 
 
 def parse_args():
@@ -46,7 +47,8 @@ def parse_args():
                     help="named configuration (2 is the one the metric is quoted on; 3 times the "
                          "pairwise cosine-distance matrix instead of the filter)")
     ap.add_argument("--tau", type=float, default=0.97)
-    ap.add_argument("--schedule", type=int, default=0, help="0 auto, 1 stepwise (streaming), 2 Gram-first")
+    ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="0 auto, 1 stepwise (streaming), 2 Gram-first in two launches, 3 Gram-first in one launch")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -358,9 +360,10 @@ def run_ours(args):
         gaf.gaf_filter_accumulate(sets[i % n_sets].grads, args.tau, ws, macro_out=macro, mask_out=mask,
                                   dist_out=dist_out, count_out=count, schedule=args.schedule)
 
-    # which schedule runs (0 = the library's choice: Gram-first up to 8 gradients) and its byte model
-    sched_used = args.schedule if args.schedule else (2 if 2 <= K <= 8 else 1)
-    model = gram_first_bytes if sched_used == 2 else schedule_bytes
+    # which schedule runs (the library says what its own choice was) and its byte model
+    step(0)
+    sched_used = gaf.gaf_last_schedule()
+    model = gram_first_bytes if sched_used in (2, 3) else schedule_bytes
     # accept pattern and byte model per input set (also a warm-up)
     masks, bytes_per_set, launches_per_step = [], [], 0
     for i in range(n_sets):
@@ -454,8 +457,8 @@ def run_ours(args):
             "config": {
                 "workload": workload_label(cfg, K, D, w0.dtype, args.tau),
                 "K": K, "D": D, "input_dtype": w0.dtype, "tau": args.tau,
-                "schedule": {0: "auto", 1: "stepwise", 2: "gram-first"}[args.schedule] +
-                            (" -> " + {1: "stepwise", 2: "gram-first"}[sched_used] if not args.schedule else ""),
+                "schedule": SCHED_NAMES[args.schedule] +
+                            (" -> " + SCHED_NAMES[sched_used] if not args.schedule else ""),
                 "parallelism": "replicas only (the path does not shard)" if world > 1 else "1 GPU",
                 "l2": f"{n_sets} rotating input sets of {grad_bytes / 1e6:.0f} MB each (inputs of a step "
                       f"exceed the 126 MB L2 and were last touched {n_sets - 1} steps earlier)"
@@ -466,11 +469,12 @@ def run_ours(args):
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak,
                 "traffic": (ncu_traffic_config2(masks, n_sets, n_launch_timed)
-                            if (cfg == 2 and sched_used == 2 and abs(args.tau - 0.97) < 1e-12) else None),
+                            if (cfg == 2 and sched_used == 3 and abs(args.tau - 0.97) < 1e-12) else None),
                 "peak_kind": f"of {peak_kind}",
-                "kernel": ("gram_small_kernel + masked_mean_kernel (whole call, both HBM-streaming)"
-                           if sched_used == 2 else "step_kernel x%d (whole call)" % launches_per_step),
-                "byte_model": ("Gram-first: ((K + c) b + 4) D" if sched_used == 2
+                "kernel": {3: "gram_fused_kernel (the whole call is this one launch)",
+                           2: "Gram kernel + masked_mean_kernel (whole call, both HBM-streaming)",
+                           1: "step_kernel x%d (whole call)" % launches_per_step}[sched_used],
+                "byte_model": ("Gram-first: ((K + c) b + 4) D" if sched_used in (2, 3)
                                else "streaming: (2b+4) + sum_t [4 + b + a_t (b+4)] + 8 + a_last b, times D"),
                 "algorithmic_bytes_per_launch": avg_bytes, "avg_launch_ms": avg_launch_ms,
                 "sustained_achieved": sustained, "sustained_frac": sustained / peak,

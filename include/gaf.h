@@ -62,29 +62,41 @@ enum {
 };
 
 /* How gaf_filter_accumulate walks the K-1 sequential decisions of Algorithm 1.
- * Both schedules produce the same mask and a bit-identical macro-gradient (the
+ * All schedules produce the same mask and a bit-identical macro-gradient (the
  * accepted gradients are always added in processing order in binary32); they
  * differ in launch structure and in how many bytes cross HBM. */
 enum {
-    GAF_SCHED_AUTO = 0,         /* the library picks (Gram-first for K <= 8) */
+    GAF_SCHED_AUTO = 0,         /* the library picks: Gram-first where a one-pass Gram kernel
+                                   applies (K <= 8, or bfloat16 up to K = 32), else stepwise.
+                                   For K <= 8 the one-launch form is taken for binary32 inputs of
+                                   at most 512 MB in all, and for bfloat16 inputs except 8
+                                   gradients of more than 1 GB in all (tensor-core Gram then). */
     GAF_SCHED_STEPWISE = 1,     /* streaming: one launch per step; each launch adds the
                                    gradient accepted at step t to the running sum and, in
                                    the same pass, takes the three dot products of the
                                    updated sum with the candidate of step t+1; decisions
                                    stay on the device */
-    GAF_SCHED_GRAM = 2          /* Gram-first: every gradient is read once to build the
+    GAF_SCHED_GRAM = 2,         /* Gram-first: every gradient is read once to build the
                                    K x K Gram matrix, the K-1 decisions are taken on it (dot
                                    products are bilinear), then the accepted gradients are
                                    read once more to write g/c.  The distances agree with
-                                   the stepwise schedule to rounding. */
+                                   the stepwise schedule to rounding.  Two launches. */
+    GAF_SCHED_GRAM_FUSED = 3    /* Gram-first as ONE launch of a co-resident grid (K <= 8): the
+                                   same two passes, with the decisions exchanged through the
+                                   workspace between them, so that part of what the first pass
+                                   read (shared memory, L2) need not cross HBM again.  Identical
+                                   outputs to GAF_SCHED_GRAM.  GAF_ERR_UNSUPPORTED for K > 8 or on
+                                   a device without cooperative launches.  Its one internal wait
+                                   is bounded: GAF_STATUS_TIMEOUT if it ever runs out. */
 };
 
 /* Bits of the device status word. */
 enum {
     GAF_STATUS_ZERO_NORM = 1,   /* some tested pair had a zero norm (distance set to 1) */
     GAF_STATUS_NONFINITE = 2,   /* some sum was NaN or Inf */
-    GAF_STATUS_TIMEOUT = 4      /* a bounded wait inside the tensor-core Gram kernel ran out;
-                                   the outputs of that call are not valid */
+    GAF_STATUS_TIMEOUT = 4      /* a bounded wait inside a kernel (tensor-core Gram pipeline,
+                                   one-launch Gram-first schedule) ran out; the outputs of that
+                                   call are not valid */
 };
 
 /* Human-readable name of a return code.  Host only; never NULL. */
@@ -295,6 +307,10 @@ int gaf_cosdist_static(const void *x, const void *y, int64_t D, int dtype,
 /* Number of kernel launches the most recent gaf_* call of this thread issued
  * (host-side counter, for benchmarks). */
 int gaf_last_launch_count(void);
+
+/* The GAF_SCHED_* value the most recent gaf_filter_accumulate call of this thread ran with
+ * (what GAF_SCHED_AUTO resolved to).  Host-side, for benchmarks and tests. */
+int gaf_last_schedule(void);
 
 #ifdef __cplusplus
 }

@@ -13,7 +13,7 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 GAF_F32, GAF_BF16 = 0, 1
-GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_GRAM = 0, 1, 2
+GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_GRAM, GAF_SCHED_GRAM_FUSED = 0, 1, 2, 3
 GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT = 1, 2, 4
 GAF_MAX_K = 64
 
@@ -25,7 +25,7 @@ EXPORTS = [
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
     "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
     "gaf_filter_accumulate_any_seed", "gaf_stream_begin", "gaf_stream_push", "gaf_stream_end",
-    "gaf_filter_accumulate_bucketed",
+    "gaf_filter_accumulate_bucketed", "gaf_last_schedule",
 ]
 
 
@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.gaf_pairwise_cosdist.argtypes = [vp, i32, i64, i32, vp, vp, vp, sz, vp]
         L.gaf_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.gaf_last_launch_count.argtypes = []
+        L.gaf_last_schedule.argtypes = []
         L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.gaf_filter_accumulate_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, vp]
         L.gaf_filter_accumulate_bucketed.argtypes = [vp, i32, i64, i32, dbl, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -298,3 +299,8 @@ def gaf_read_status(workspace: torch.Tensor) -> int:
 
 def gaf_last_launch_count() -> int:
     return lib().gaf_last_launch_count()
+
+
+def gaf_last_schedule() -> int:
+    """The GAF_SCHED_* value the latest gaf_filter_accumulate call of this thread ran with."""
+    return lib().gaf_last_schedule()

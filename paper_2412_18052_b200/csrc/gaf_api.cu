@@ -20,6 +20,7 @@ namespace {
 using namespace gaf;
 
 thread_local int g_launches = 0;
+thread_local int g_schedule = 0;       // what the latest gaf_filter_accumulate resolved AUTO to
 
 struct DeviceInfo {
     int sms = 0;
@@ -57,11 +58,14 @@ int stream_grid(int64_t D, int threads, int sms) {
     return int(need < cap ? need : cap);
 }
 
-// Which Gram kernel: bfloat16 with up to 32 gradients goes to the tensor cores, except that
-// with at most 8 gradients and a short vector the one-launch register-tiled kernel wins.
-constexpr int64_t kTcMinSmallK = int64_t(1) << 22;
+// Which Gram kernel.  The tensor-core kernel pays off from 8 bfloat16 gradients on: with fewer, most
+// of each 128-row MMA tile is padding and the register-tiled kernel is faster at every length
+// (measured: 4 gradients of 5e8 elements, 1.85 ms against 1.41 ms).  With exactly 8 it wins only
+// once the vectors are long enough for the one-launch schedule to have lost its edge.
+constexpr int64_t kTcMinBytesK8 = int64_t(1) << 30;
 bool use_tensor_gram(int K, int64_t D, int dtype) {
-    return dtype == GAF_BF16 && K >= 2 && K <= kTcMaxK && (K > kGsMaxK || D >= kTcMinSmallK);
+    if (dtype != GAF_BF16 || K < kGsMaxK || K > kTcMaxK) return false;
+    return K > kGsMaxK || int64_t(K) * 2 * D > kTcMinBytesK8;
 }
 bool use_small_gram(int K, int64_t D, int dtype) {
     return K >= 2 && K <= kGsMaxK && !use_tensor_gram(K, D, dtype);
@@ -168,12 +172,16 @@ int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
 }
 
 // One-launch form of the Gram-first schedule (gaf_fused.cuh).  Returns GAF_OK when it was
-// launched, -1 when this device or size does not allow it (the caller then takes the two-launch
-// form), or an error code.
-int g_carveout_pct = -1;
-int g_keep_l2_pct = 10;                 // share of L2 the Gram pass asks to keep for the second pass
-int g_park_rounds_max = 2;
-constexpr int64_t kFusedMaxInputBytes = int64_t(1) << 30;   // beyond this nothing stays on chip anyway
+// launched, GAF_ERR_UNSUPPORTED when this device or K does not allow it, or an error code.
+constexpr int kKeepL2Pct = 10;          // share of L2 the Gram pass asks to keep for the second pass
+                                        // (measured: larger shares slow both passes down)
+// Shared memory of one SM given to parked rounds.  The rest of the L1/shared array stays L1, which the
+// loads in flight need: beyond about 60 % shared memory both passes lose more than parking gains.
+constexpr int kParkBytesPerSm = 128 << 10;
+// AUTO takes the one-launch form for binary32 inputs up to this many bytes in all: beyond, what stays
+// on chip between the passes is a negligible share and the two-launch form is as fast or slightly
+// faster.  For bfloat16 the one-launch form stays ahead at every length measured.
+constexpr int64_t kFusedMaxInputBytesF32 = int64_t(512) << 20;
 
 template <typename T, int KT>
 int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st) {
@@ -181,29 +189,28 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
     // CTAs per SM by registers alone, then as many parked rounds as shared memory allows
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kGsThreads, 0) != cudaSuccess || occ < 1)
-        return -1;
+        return GAF_ERR_UNSUPPORTED;
     if (occ > 2) occ = 2;
     cudaFuncAttributes fa{};
     if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return GAF_ERR_CUDA;
     const int round_bytes = KT * kGsThreads * 16;
     int64_t budget = di.smem_per_sm / occ - 1024 - int64_t(fa.sharedSizeBytes);
     if (budget > di.smem_per_cta_max - int64_t(fa.sharedSizeBytes)) budget = di.smem_per_cta_max - int64_t(fa.sharedSizeBytes);
-    int park = budget > 0 ? int(budget / round_bytes) : 0;
-    if (park > g_park_rounds_max) park = g_park_rounds_max;
+    if (budget > kParkBytesPerSm / occ) budget = kParkBytesPerSm / occ;
+    const int park = budget > 0 ? int(budget / round_bytes) : 0;
     const int dyn = park * round_bytes;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
         return GAF_ERR_CUDA;
     {
         // shared memory share of the L1/shared array: what the CTAs of one SM need, no more (the rest is L1)
-        int pct = g_carveout_pct >= 0 ? g_carveout_pct
-                                      : int((int64_t(dyn + fa.sharedSizeBytes + 1024) * occ * 100 + di.smem_per_sm - 1) / di.smem_per_sm);
+        int pct = int((int64_t(dyn + fa.sharedSizeBytes + 1024) * occ * 100 + di.smem_per_sm - 1) / di.smem_per_sm);
         if (pct > 100) pct = 100;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, pct) != cudaSuccess)
             return GAF_ERR_CUDA;
     }
     int occ2 = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ2, kernel, kGsThreads, dyn) != cudaSuccess || occ2 < 1)
-        return -1;
+        return GAF_ERR_UNSUPPORTED;
     if (occ2 < occ) occ = occ2;
     int64_t grid = int64_t(di.sms) * occ;
     if (grid > kGsMaxCtas) grid = kGsMaxCtas;
@@ -213,7 +220,7 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
     a.park_rounds = park;
     // the last stretch is asked to stay in L2 for the second pass
     const int64_t per_elem = int64_t(KT) * int64_t(sizeof(T));
-    const int64_t keep_elems = int64_t(di.l2_bytes) * g_keep_l2_pct / 100 / per_elem;
+    const int64_t keep_elems = int64_t(di.l2_bytes) * kKeepL2Pct / 100 / per_elem;
     a.keep_from = a.D > keep_elems ? a.D - keep_elems : 0;
     void *params[] = {&a};
     const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kernel), dim3(int(grid)),
@@ -225,8 +232,7 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
 
 template <typename T>
 int launch_gram_fused(GramFusedArgs &a, int K, const DeviceInfo &di, cudaStream_t st) {
-    if (!di.cooperative || g_park_rounds_max < 0) return -1;
-    if (int64_t(K) * int64_t(sizeof(T)) * a.D > kFusedMaxInputBytes) return -1;
+    if (!di.cooperative) return GAF_ERR_UNSUPPORTED;
     switch (K) {
         case 2: return launch_gram_fused_kt<T, 2>(a, di, st);
         case 3: return launch_gram_fused_kt<T, 3>(a, di, st);
@@ -235,7 +241,7 @@ int launch_gram_fused(GramFusedArgs &a, int K, const DeviceInfo &di, cudaStream_
         case 6: return launch_gram_fused_kt<T, 6>(a, di, st);
         case 7: return launch_gram_fused_kt<T, 7>(a, di, st);
         case 8: return launch_gram_fused_kt<T, 8>(a, di, st);
-        default: return -1;
+        default: return GAF_ERR_UNSUPPORTED;
     }
 }
 
@@ -244,7 +250,8 @@ int launch_gram_fused(GramFusedArgs &a, int K, const DeviceInfo &di, cudaStream_
 template <typename T>
 int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double tau, const int32_t *ord,
                       float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
-                      int32_t *seed_out, unsigned char *base, const DeviceInfo &di, cudaStream_t st) {
+                      int32_t *seed_out, unsigned char *base, const DeviceInfo &di, bool one_launch,
+                      cudaStream_t st) {
     const int sms = di.sms;
     Control *ctl = reinterpret_cast<Control *>(base);
     RingArgs ring{};
@@ -258,8 +265,8 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     double *gram_by_index = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K));
     double *gram_by_step = reinterpret_cast<double *>(base + kExtraOffset + gram_partials_bytes(K) +
                                                       gram_matrix_bytes(K));
-    if (use_small_gram(K, D, dtype)) {
-        // short calls: both passes in one co-resident launch
+    if (one_launch) {
+        if (K < 2 || K > kGsMaxK) return GAF_ERR_UNSUPPORTED;
         GramFusedArgs f{};
         for (int t = 0; t < K; ++t) f.g[t] = g[ord[t]];
         f.D = D; f.out = macro_out;
@@ -267,15 +274,15 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
         f.gram = gram_by_step;
         f.replay = r;
         f.ring = ring;
-        const int frc = launch_gram_fused<T>(f, K, di, st);
-        if (frc >= 0) return frc;
-
+        return launch_gram_fused<T>(f, K, di, st);
+    }
+    if (use_small_gram(K, D, dtype)) {
         GramSmallArgs a{};
         for (int t = 0; t < K; ++t) a.g[t] = g[ord[t]];
         a.D = D;
         // how much of the tail of the Gram pass should stay in L2 for the masked-mean pass
         const int64_t per_elem = int64_t(K) * int64_t(sizeof(T));
-        const int64_t keep_elems = int64_t(di.l2_bytes) * g_keep_l2_pct / 100 / per_elem;
+        const int64_t keep_elems = int64_t(di.l2_bytes) * kKeepL2Pct / 100 / per_elem;
         a.keep_from = D > keep_elems ? D - keep_elems : 0;
         a.partials = reinterpret_cast<double *>(base + kExtraOffset);
         a.gram = gram_by_step;
@@ -304,6 +311,12 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     ++g_launches;
     if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
+}
+
+// Whether the library's own choice is the one-launch form of the Gram-first schedule.
+bool auto_one_launch(int K, int64_t D, int dtype, const DeviceInfo &di) {
+    return di.cooperative && use_small_gram(K, D, dtype) &&
+           (dtype == GAF_BF16 || int64_t(K) * 4 * D <= kFusedMaxInputBytesF32);
 }
 
 int check_workspace(const void *ws, size_t have, size_t need) {
@@ -390,6 +403,7 @@ const char *gaf_error_string(int code) {
 }
 
 int gaf_last_launch_count(void) { return g_launches; }
+int gaf_last_schedule(void) { return g_schedule; }
 
 int gaf_workspace_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {
     if (!bytes_out || K < 1 || K > GAF_MAX_K || D < 0) return GAF_ERR_ARG;
@@ -433,7 +447,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     g_launches = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if ((!macro_out && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
-    if (schedule < GAF_SCHED_AUTO || schedule > GAF_SCHED_GRAM) return GAF_ERR_ARG;
+    if (schedule < GAF_SCHED_AUTO || schedule > GAF_SCHED_GRAM_FUSED) return GAF_ERR_ARG;
     if (tau != tau) return GAF_ERR_ARG;
     if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
     int32_t ord[GAF_MAX_K];
@@ -466,16 +480,20 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
         // Gram-first moves fewer bytes whenever its one-pass Gram kernel applies
         const bool ws_ok = workspace_bytes >= kExtraOffset + pairwise_extra_bytes(K);
         const bool fast_gram = K >= 2 && (K <= kGsMaxK || use_tensor_gram(K, D, dtype));
-        schedule = (fast_gram && ws_ok) ? GAF_SCHED_GRAM : GAF_SCHED_STEPWISE;
+        schedule = (fast_gram && ws_ok) ? (auto_one_launch(K, D, dtype, di) ? GAF_SCHED_GRAM_FUSED : GAF_SCHED_GRAM)
+                                        : GAF_SCHED_STEPWISE;
     }
-    if (schedule == GAF_SCHED_GRAM && K >= 2) {
+    if (K == 1) schedule = GAF_SCHED_STEPWISE;          // one gradient: it is the seed and the result
+    g_schedule = schedule;
+    if (schedule == GAF_SCHED_GRAM || schedule == GAF_SCHED_GRAM_FUSED) {
         if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K)))
             return rc;
+        const bool one_launch = schedule == GAF_SCHED_GRAM_FUSED;
         return dtype == GAF_F32
             ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                       count_out, nullptr, base, di, st)
+                                       count_out, nullptr, base, di, one_launch, st)
             : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                               count_out, nullptr, base, di, st);
+                                               count_out, nullptr, base, di, one_launch, st);
     }
     return dtype == GAF_F32
         ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
@@ -522,9 +540,9 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
     }
     return dtype == GAF_F32
         ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out, count_out,
-                                   seed_out, base, di, st)
+                                   seed_out, base, di, auto_one_launch(K, D, dtype, di), st)
         : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                           count_out, seed_out, base, di, st);
+                                           count_out, seed_out, base, di, auto_one_launch(K, D, dtype, di), st);
 }
 
 int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, int dtype, double tau,

@@ -234,17 +234,20 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     if (n < 0) return;
     const float cdiv = (float)n;
 
-    // ---- pass 2a: the rounds that were not parked, last first (the most recently read lines
-    //      are the ones still in L2), two rounds in flight per thread ----
+    // ---- pass 2a: the rounds that were not parked, last first (what pass 1 read last is what
+    //      L2 still holds), two rounds in flight per thread ----
     constexpr int U = 2;
     for (int64_t j0 = rounds - 1; j0 >= parked_rounds; j0 -= U) {
+        int64_t ju[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) ju[u] = j0 - u >= parked_rounds ? j0 - u : -1;
         int64_t q[U];
         bool ok[U];
         uint4 w[U][KT];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            q[u] = warp_first + (j0 - u) * stride + lane;
-            ok[u] = (j0 - u) >= parked_rounds && q[u] < n_vec;
+            q[u] = warp_first + ju[u] * stride + lane;
+            ok[u] = ju[u] >= 0 && q[u] < n_vec;
 #pragma unroll
             for (int i = 0; i < KT; ++i)
                 if (ok[u] && i < n) w[u][i] = ld16_policy(list[i] + q[u] * N, pol_first);

@@ -251,7 +251,7 @@ struct GramSmallArgs {
 // 16-byte read-only load with an explicit L2 eviction policy.
 __device__ __forceinline__ uint4 ld16_policy(const void *p, uint64_t policy) {
     uint4 r;
-    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
                  : "l"(p), "l"(policy));
     return r;

@@ -12,8 +12,8 @@ from parity import check_any_seed, check_bucketed, check_cosdist, check_filter, 
 
 pytestmark = pytest.mark.gpu
 
-SCHEDULES = [gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_GRAM]
-SCHED_IDS = ["stepwise", "gram"]
+SCHEDULES = [gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_GRAM, gaf.GAF_SCHED_GRAM_FUSED]
+SCHED_IDS = ["stepwise", "gram", "gram-one-launch"]
 DTYPES = ["f32", "bf16"]
 
 
@@ -148,6 +148,15 @@ def test_filter_degenerate_inputs(ws, schedule):
 def test_filter_maximum_k(ws, schedule):
     K = gaf.binding.GAF_MAX_K
     w = _mix(K, 10_007, "bf16", seed=64)
+    if schedule == gaf.GAF_SCHED_GRAM_FUSED:
+        # the one-launch form handles up to 8 gradients and says so beyond
+        with pytest.raises(gaf.GafError) as e:
+            gaf.gaf_filter_accumulate(w.grads, 0.97, ws, schedule=schedule)
+        assert e.value.code == 7
+        w = _mix(8, 10_007, "bf16", seed=64)
+        r = check_filter(w.grads, 0.97, ws, schedule=schedule)
+        assert 1 < r["count"] < 8
+        return
     r = check_filter(w.grads, 0.97, ws, schedule=schedule)
     assert 1 < r["count"] < K
 
@@ -178,11 +187,16 @@ def test_schedules_agree(ws):
     w = _mix(5, 2_000_003, "bf16", seed=12)
     a = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_STEPWISE)
     a = [t.clone() for t in a]
-    for other in (gaf.GAF_SCHED_GRAM, gaf.GAF_SCHED_AUTO):
+    outs = {}
+    for other in (gaf.GAF_SCHED_GRAM, gaf.GAF_SCHED_GRAM_FUSED, gaf.GAF_SCHED_AUTO):
         b = gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=other)
         assert torch.equal(a[1], b[1]) and torch.equal(a[3], b[3])
         assert float((a[2] - b[2]).abs().max()) < 1e-6
         assert torch.equal(a[0], b[0])       # element arithmetic is identical in every schedule
+        outs[other] = [t.clone() for t in b]
+    # the two forms of the Gram-first schedule take the same sums in the same order
+    for x, y in zip(outs[gaf.GAF_SCHED_GRAM], outs[gaf.GAF_SCHED_GRAM_FUSED]):
+        assert torch.equal(x, y)
 
 
 def test_filter_host_entry_point(ws):
@@ -211,7 +225,10 @@ def test_filter_random_cases(ws):
         dtype = "bf16" if rng.rand() < 0.5 else "f32"
         tau = float(rng.choice([0.3, 0.8, 0.97, 1.0, 1.1, 1.6]))
         order = [int(x) for x in rng.permutation(K)] if rng.rand() < 0.5 else None
-        schedule = int(rng.choice([gaf.GAF_SCHED_AUTO, gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_GRAM]))
+        schedule = int(rng.choice([gaf.GAF_SCHED_AUTO, gaf.GAF_SCHED_STEPWISE, gaf.GAF_SCHED_GRAM,
+                                   gaf.GAF_SCHED_GRAM_FUSED]))
+        if schedule == gaf.GAF_SCHED_GRAM_FUSED and K > 8:
+            schedule = gaf.GAF_SCHED_GRAM
         w = _mix(K, D, dtype, seed=5000 + case, sigma=float(rng.choice([1e-3, 1.0, 30.0])))
         check_filter(w.grads, tau, ws, order=order, schedule=schedule, expect_status=None)
 
@@ -227,6 +244,7 @@ def test_gram_loop_ends_inside_a_warp_at_the_flush_period(ws, dtype):
         D = (threads * 15 + extra) * per_vec + 3
         w = _mix(3, D, dtype, seed=77, rho=[0.7, 0.5, -0.4])
         check_filter(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_GRAM)
+        check_filter(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED)
         check_pairwise(w.grads, ws)
 
 
