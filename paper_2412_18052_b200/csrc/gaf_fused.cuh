@@ -172,9 +172,15 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     flush();
     __syncthreads();
     if (tid < NP) {
-        double s = 0.0;
-        for (int w = 0; w < kGsThreads / 32; ++w) s += sacc[w][tid];
-        a.partials[(size_t)tid * kGsPartialStride + blockIdx.x] = s;
+        // the 16 warps' sums in four short chains (a fixed order, so still reproducible)
+        double s4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            s4[c] = sacc[4 * c][tid];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) s4[c] += sacc[4 * c + w][tid];
+        }
+        a.partials[(size_t)tid * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     }
     __threadfence();
     __syncthreads();
@@ -201,7 +207,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
             ring_replay_on_gram(a.ring, sgram, ring_count, ring_bits, notice);
         } else {
             __shared__ ReplayTable table;
-            replay_on_gram_parallel(a.replay, sgram, table, [&](unsigned long long bits) { notice(-1, bits); });
+            replay_on_gram_parallel<KT>(a.replay, sgram, table, [&](unsigned long long bits) { notice(-1, bits); });
         }
     }
     if (tid == 0) {

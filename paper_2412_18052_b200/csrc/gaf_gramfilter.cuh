@@ -94,26 +94,32 @@ struct ReplayTable {
 struct NoEarlyBits {
     __device__ __forceinline__ void operator()(unsigned long long) const {}
 };
-template <typename Early = NoEarlyBits>
+template <int KT, typename Early = NoEarlyBits>
 __device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, const double *gram, ReplayTable &tb,
                                                         Early early = Early()) {
-    const int K = r.K, tid = threadIdx.x;
-    const int cases = (1 << (K - 1)) - 1;
+    constexpr int K = KT;
+    const int tid = threadIdx.x;
+    constexpr int cases = (1 << (K - 1)) - 1;
     if (tid < cases) {
         const int t = 32 - __clz(tid + 1);                      // tid + 1 in [2^(t-1), 2^t)
         const unsigned int m = (unsigned int)(tid + 1) - (1u << (t - 1));
-        auto in = [&](int v) { return v == 0 || ((m >> (v - 1)) & 1u); };   // step v accepted in this case
+        // step v accepted in this case (bits of m at and above t-1 are zero)
+        auto in = [&](int v) { return v == 0 || ((m >> (v - 1)) & 1u); };
+        // Branch-free (neighbouring lanes hold different cases): a gradient that is not in the case
+        // contributes an added 0.0, which leaves a binary64 sum unchanged, and its update of |g|^2
+        // is computed and dropped.
         double na = gram[0];
-        for (int u = 1; u < t; ++u)
-            if (in(u)) {
-                double pu = 0.0;
-                for (int v = 0; v < u; ++v)
-                    if (in(v)) pu += gram[v * K + u];
-                na = na + 2.0 * pu + gram[u * K + u];
-            }
+#pragma unroll
+        for (int u = 1; u < K - 1; ++u) {
+            double pu = 0.0;
+#pragma unroll
+            for (int v = 0; v < u; ++v) pu += in(v) ? gram[v * K + u] : 0.0;
+            const double grown = na + 2.0 * pu + gram[u * K + u];
+            na = in(u) ? grown : na;
+        }
         double p = 0.0;
-        for (int v = 0; v < t; ++v)
-            if (in(v)) p += gram[v * K + t];
+#pragma unroll
+        for (int v = 0; v < K - 1; ++v) p += (v < t && in(v)) ? gram[v * K + t] : 0.0;
         int status = 0;
         const double d = cosine_distance(p, na, gram[t * K + t], &status);
         tb.d[tid] = d; tb.p[tid] = p; tb.na[tid] = na;
@@ -413,9 +419,15 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __syncthreads();
     if (threadIdx.x < NP) {
-        double s = 0.0;
-        for (int w = 0; w < kGsThreads / 32; ++w) s += sacc[w][threadIdx.x];
-        a.partials[(size_t)threadIdx.x * kGsPartialStride + blockIdx.x] = s;
+        // the 16 warps' sums in four short chains (a fixed order, so still reproducible)
+        double s4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            s4[c] = sacc[4 * c][threadIdx.x];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) s4[c] += sacc[4 * c + w][threadIdx.x];
+        }
+        a.partials[(size_t)threadIdx.x * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     }
     __threadfence();
     __syncthreads();
@@ -440,7 +452,7 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
     }
     if (a.pair_dist_out == nullptr) {
         __shared__ ReplayTable table;
-        replay_on_gram_parallel(a.replay, sgram, table);
+        replay_on_gram_parallel<KT>(a.replay, sgram, table);
         return;
     }
     // pairwise mode: Eq. 4 for every pair
