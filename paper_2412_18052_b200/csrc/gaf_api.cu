@@ -135,8 +135,18 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
         ++g_launches;
     }
-    gram_finish_kernel<<<pairs, 64 * kFinishParts, 0, st>>>(a);
-    ++g_launches;
+    {
+        // programmatic dependent launch: the finishing blocks are placed while the Gram kernel winds down
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(pairs); cfg.blockDim = dim3(64 * kFinishParts); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const cudaError_t err = cudaLaunchKernelEx(&cfg, gram_finish_kernel, a);
+        ++g_launches;
+        if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+    }
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }
 

@@ -340,6 +340,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
         if (threadIdx.x == 0) atomicOr(&a.ctl->status, kStatusTimeoutBit);
         return;
     }
+    // the streaming part of this CTA is over: the finishing kernel, launched as a programmatic
+    // dependent, may be placed now; it still waits for this whole grid before it reads the partials
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles <= 32 KB)
     double *red = reinterpret_cast<double *>(tiles);
     if (warp < 4) {

@@ -149,6 +149,9 @@ __global__ void __launch_bounds__(64 * kFinishParts) gram_finish_kernel(GramArgs
     int ti, tj;
     tile_pair(blockIdx.x, a.tiles, ti, tj);
     const int p = threadIdx.x & 63, chain = threadIdx.x >> 6;
+    // launched as a programmatic dependent of the Gram kernel: wait until that grid has completed
+    // and its partial sums are visible (a no-op in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     {
         const int per = (a.slices + kFinishParts - 1) / kFinishParts;
         const int lo = chain * per, hi = min(a.slices, lo + per);
