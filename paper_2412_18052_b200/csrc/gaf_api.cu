@@ -334,6 +334,19 @@ int check_workspace(const void *ws, size_t have, size_t need) {
     return GAF_OK;
 }
 
+// Launch `kernel` as a programmatic dependent of the launch before it on the stream: its blocks may be
+// placed while that grid winds down; the kernel itself waits (griddepcontrol.wait) for that grid.
+template <typename Args>
+cudaError_t launch_dependent(void (*kernel)(Args), int grid, int threads, cudaStream_t st, const Args &args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args);
+}
+
 template <typename T>
 int launch_stepwise(const void *const *g, int K, int64_t D, double tau, const int32_t *ord,
                     float *macro_out, uint8_t *mask_out, float *dist_out, int32_t *count_out,
@@ -354,11 +367,17 @@ int launch_stepwise(const void *const *g, int K, int64_t D, double tau, const in
     ++g_launches;
     for (int t = 1; t <= K - 2; ++t) {
         a.t = t; a.g_cur = g[ord[t]]; a.g_next = g[ord[t + 1]]; a.i_next = ord[t + 1];
-        step_kernel<T, kMid><<<grid, kStepThreads, 0, st>>>(a);
+        if (launch_dependent(step_kernel<T, kMid>, grid, kStepThreads, st, a) != cudaSuccess) {
+            cudaGetLastError();
+            return GAF_ERR_CUDA;
+        }
         ++g_launches;
     }
     a.t = K - 1; a.g_cur = g[ord[K - 1]]; a.g_next = nullptr; a.i_next = -1;
-    step_kernel<T, kLast><<<grid, kStepThreads, 0, st>>>(a);
+    if (launch_dependent(step_kernel<T, kLast>, grid, kStepThreads, st, a) != cudaSuccess) {
+        cudaGetLastError();
+        return GAF_ERR_CUDA;
+    }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }

@@ -72,6 +72,9 @@ __global__ void __launch_bounds__(kStepThreads, 2) step_kernel(StepArgs a) {
 
     int accept = 0, count = 1;
     if (MODE == kMid || MODE == kLast) {
+        // launched as a programmatic dependent of the previous step's launch: its blocks are placed
+        // while that grid winds down, and wait here until it has completed and its decision is visible
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         accept = *reinterpret_cast<volatile int *>(&a.ctl->decision[a.t]);
         count = *reinterpret_cast<volatile int *>(&a.ctl->count);
     }
@@ -132,6 +135,8 @@ __global__ void __launch_bounds__(kStepThreads, 2) step_kernel(StepArgs a) {
     }
 
     if (MODE == kFirst || MODE == kMid) {
+        // the streaming part of this CTA is over: the next step's launch may start placing blocks
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         Sums3 blk = block_reduce(s, scratch);
         finalize_step(a, blk, a.t + 1);
     } else if (MODE == kLast) {
