@@ -9,6 +9,7 @@
 #include "gaf_bucketed.cuh"
 #include "gaf_device.cuh"
 #include "gaf_fused.cuh"
+#include "gaf_gram_panel.cuh"
 #include "gaf_gram_tc.cuh"
 #include "gaf_gramfilter.cuh"
 #include "gaf_pairwise.cuh"
@@ -63,6 +64,7 @@ int stream_grid(int64_t D, int threads, int sms) {
 // (measured: 4 gradients of 5e8 elements, 1.85 ms against 1.41 ms).  With exactly 8 it wins only
 // once the vectors are long enough for the one-launch schedule to have lost its edge.
 constexpr int64_t kTcMinBytesK8 = int64_t(1) << 30;
+constexpr int kPanelAutoMaxK = 32;
 bool use_tensor_gram(int K, int64_t D, int dtype) {
     if (dtype != GAF_BF16 || K < kGsMaxK || K > kTcMaxK) return false;
     return K > kGsMaxK || int64_t(K) * 2 * D > kTcMinBytesK8;
@@ -123,16 +125,38 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         gram_tc_kernel<<<a.slices, kTcThreads, dyn, st>>>(t);
         ++g_launches;
     } else {
-        // D-slices: fill the machine about twice over all tile pairs, never more than there is work
-        int64_t slices = (int64_t(sms) * 2 + pairs - 1) / pairs;
-        const int64_t work = (D / 4 + kGramThreads - 1) / kGramThreads;
+        // CUDA cores, every gradient read once: one warp per tile pair, panels of D through shared memory
+        GramPanelArgs pa{};
+        for (int i = 0; i < K; ++i) pa.g[i] = grads[i];
+        pa.K = K; pa.D = D; pa.tiles = a.tiles; pa.pairs = pairs;
+        const int groups = (pairs + kPanelMaxWarps - 1) / kPanelMaxWarps;
+        pa.pairs_per_cta = (pairs + groups - 1) / groups;
+        // A panel is at most 32 KB: 2 KB of every row up to 16 (padded) rows, 1 KB up to 32, 512 bytes
+        // beyond.  With 3 or 6 tile pairs, 4 or 2 warps share a pair.
+        const int shift = a.tiles <= 2 ? 7 : (a.tiles <= 4 ? 6 : 5);
+        const int wpp = a.tiles <= 2 ? 4 : (a.tiles == 3 ? 2 : 1);
+        pa.partials = a.partials; pa.ctl = a.ctl;
+        const int threads = 32 * pa.pairs_per_cta * wpp;
+        const int row_bytes = 16 << shift;
+        const int dyn = kPanelStages * a.tiles * 8 * row_bytes;
+        void (*kernel)(GramPanelArgs) = nullptr;
+        if (dtype == GAF_F32)
+            kernel = shift == 7 ? gram_panel_kernel<float, 7, 4>
+                   : (shift == 6 ? (wpp == 2 ? gram_panel_kernel<float, 6, 2> : gram_panel_kernel<float, 6, 1>)
+                                 : gram_panel_kernel<float, 5, 1>);
+        else
+            kernel = shift == 7 ? gram_panel_kernel<__nv_bfloat16, 7, 4>
+                   : (shift == 6 ? (wpp == 2 ? gram_panel_kernel<__nv_bfloat16, 6, 2> : gram_panel_kernel<__nv_bfloat16, 6, 1>)
+                                 : gram_panel_kernel<__nv_bfloat16, 5, 1>);
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+            return GAF_ERR_CUDA;
+        const int64_t chunk_elems = row_bytes / int64_t(elem_bytes(dtype));
+        const int64_t work = (D + chunk_elems - 1) / chunk_elems;
+        int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;      // one CTA per SM
         if (slices > work) slices = work;
-        if (slices > kGramMaxSlices) slices = kGramMaxSlices;
         if (slices < 1) slices = 1;
         a.slices = int(slices);
-        dim3 grid(a.slices, pairs);
-        if (dtype == GAF_F32) gram_tile_kernel<float><<<grid, kGramThreads, 0, st>>>(a);
-        else gram_tile_kernel<__nv_bfloat16><<<grid, kGramThreads, 0, st>>>(a);
+        kernel<<<dim3(a.slices, groups), threads, dyn, st>>>(pa);
         ++g_launches;
     }
     {
@@ -508,7 +532,9 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     if (schedule == GAF_SCHED_AUTO) {
         // Gram-first moves fewer bytes whenever its one-pass Gram kernel applies
         const bool ws_ok = workspace_bytes >= kExtraOffset + pairwise_extra_bytes(K);
-        const bool fast_gram = K >= 2 && (K <= kGsMaxK || use_tensor_gram(K, D, dtype));
+        // (the general CUDA-core Gram kernel beats the stepwise schedule up to 32 binary32 gradients)
+        const bool fast_gram = K >= 2 && (K <= kGsMaxK || use_tensor_gram(K, D, dtype) ||
+                                          (dtype == GAF_F32 && K <= kPanelAutoMaxK));
         schedule = (fast_gram && ws_ok) ? (auto_one_launch(K, D, dtype, di) ? GAF_SCHED_GRAM_FUSED : GAF_SCHED_GRAM)
                                         : GAF_SCHED_STEPWISE;
     }

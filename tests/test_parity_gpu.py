@@ -406,6 +406,36 @@ def test_pairwise_small(ws, dtype):
     check_pairwise(w.grads, ws)
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("K", [10, 16, 24, 32, 40, 48, 64])
+def test_pairwise_general_kernel_shapes(ws, dtype, K):
+    """The general CUDA-core Gram kernel in each of its shapes (warps sharing a tile pair, one warp
+    per pair, tile pairs split over groups of CTAs): several panels per CTA and a ragged last one."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for D in (sms * 512 * 3 + 1234 + 3, 100_001):
+        w = _mix(K, D, dtype, seed=300 + K)
+        check_pairwise(w.grads, ws)
+
+
+def test_auto_schedule_choice(ws):
+    """What GAF_SCHED_AUTO resolves to (gaf_last_schedule), shape by shape."""
+    cases = [(1, 1000, "f32", gaf.GAF_SCHED_STEPWISE), (4, 100_000, "f32", gaf.GAF_SCHED_GRAM_FUSED),
+             (8, 100_000, "bf16", gaf.GAF_SCHED_GRAM_FUSED), (6, 50_000, "bf16", gaf.GAF_SCHED_GRAM_FUSED),
+             (9, 50_000, "f32", gaf.GAF_SCHED_GRAM), (32, 20_000, "f32", gaf.GAF_SCHED_GRAM),
+             (33, 20_000, "f32", gaf.GAF_SCHED_STEPWISE), (16, 50_000, "bf16", gaf.GAF_SCHED_GRAM),
+             (33, 20_000, "bf16", gaf.GAF_SCHED_STEPWISE)]
+    for K, D, dtype, want in cases:
+        w = _mix(K, D, dtype, seed=11)
+        gaf.gaf_filter_accumulate(w.grads, 0.97, ws)
+        assert gaf.gaf_last_schedule() == want, (K, D, dtype, gaf.gaf_last_schedule())
+    # 8 binary32 gradients of more than 512 MB in all: Gram-first in two launches
+    big = [torch.zeros(17_000_000, device="cuda") for _ in range(8)]
+    for i, g in enumerate(big):
+        g[i::8] = 1.0
+    gaf.gaf_filter_accumulate(big, 0.97, ws)
+    assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM
+
+
 def test_pairwise_zero_norm_row(ws):
     w = _mix(4, 5001, "f32", seed=2)
     w.grads[2].zero_()
