@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--D", type=int, default=None,
                     help="shorter vectors of the same recipe (for profiler captures, which must stay small); "
                          "the line then says so in config.workload")
+    ap.add_argument("--K", type=int, default=None, help="pairwise workload only: another number of gradients")
+    ap.add_argument("--fp32", action="store_true", help="pairwise workload only: binary32 inputs (same recipe)")
     ap.add_argument("--tau", type=float, default=0.97)
     ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2, 3],
                     help="0 auto, 1 stepwise (streaming), 2 Gram-first in two launches, 3 Gram-first in one launch")
@@ -290,9 +292,12 @@ def run_pairwise(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(0)
-    w = workloads.config(3, device="cuda:0")
+    w = workloads.config(3, device="cuda:0", K=args.K, D=args.D)
+    named = args.K is None and args.D is None and not args.fp32
+    if args.fp32:
+        w = workloads.mixture(w.K, w.D, "f32", w.rho, w.seed, device="cuda:0")
     K, D, b = w.K, w.D, w.elem_bytes
-    ws = gaf.new_workspace(K, D, gaf.GAF_BF16, device="cuda:0")
+    ws = gaf.new_workspace(K, D, gaf.GAF_F32 if args.fp32 else gaf.GAF_BF16, device="cuda:0")
     dist_out = torch.empty(K, K, dtype=torch.float32, device="cuda:0")
     gram = torch.empty(K, K, dtype=torch.float64, device="cuda:0")
 
@@ -323,13 +328,17 @@ def run_pairwise(args):
     line = {
         "metric": "gaf_pairwise_cosdist micro-gradient GB/s", "value": achieved, "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32 (tensor cores), f64 sums",
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 products, f64 sums" if (args.fp32 or K > 32) else "bf16 x bf16 -> f32 (tensor cores), f64 sums",
         "data": "synthetic",
-        "config": {"workload": f"configuration 3: pairwise matrix, K={K}, D={D}, bf16 inputs", "K": K, "D": D,
+        "config": {"workload": f"configuration 3: pairwise matrix, K={K}, D={D}, {w.dtype} inputs" +
+                               ("" if named else " (NOT the named configuration: size or type overridden)"),
+                   "K": K, "D": D,
                    "l2": f"inputs of one call ({in_bytes / 1e6:.0f} MB) exceed the 126 MB L2"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_kind": f"of {peak_kind}",
-                     "kernel": "gram_tc_kernel + gram_finish_kernel (whole call)",
+                     "kernel": ("gram_tc_kernel" if (not args.fp32 and 8 < K <= 32) else
+                                "gram_panel_kernel" if K > 8 else "gram_small_kernel") + " + finishing (whole call)",
                      "byte_model": "every gradient read once: K b D", "algorithmic_bytes_per_launch": in_bytes},
         "e2e": None, "gpu_launches": launches * args.steps, "clocks": clocks, "cpu_baseline": None,
     }
