@@ -67,7 +67,7 @@ enum {
  * differ in launch structure and in how many bytes cross HBM. */
 enum {
     GAF_SCHED_AUTO = 0,         /* the library picks: Gram-first where a one-pass Gram kernel
-                                   pays off (K <= 32), else stepwise.
+                                   pays off (K <= 32; bfloat16: K <= 64), else stepwise.
                                    For K <= 8 the one-launch form is taken for binary32 inputs of
                                    at most 512 MB in all, and for bfloat16 inputs except 8
                                    gradients of more than 1 GB in all (tensor-core Gram then). */

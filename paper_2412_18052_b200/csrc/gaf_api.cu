@@ -111,7 +111,7 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         // tensor cores: one CTA per SM, each with a contiguous slice of D
         GramTcArgs t{};
         for (int i = 0; i < K; ++i) t.g[i] = grads[i];
-        t.K = K; t.Kp = K <= 8 ? 8 : (K <= 16 ? 16 : 32); t.D = D;
+        t.K = K; t.Kp = K <= 8 ? 8 : (K <= 16 ? 16 : (K <= 32 ? 32 : 64)); t.D = D;
         t.partials = a.partials; t.tiles = a.tiles; t.ctl = a.ctl;
         const int64_t unit = (128 / t.Kp) * 64 * kTcSub;
         const int64_t units = (D + unit - 1) / unit;
@@ -120,9 +120,10 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         if (slices < 1) slices = 1;
         a.slices = int(slices);
         const int dyn = kTcStages * kTcStageBytes + 1024;
-        if (cudaFuncSetAttribute(gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+        auto kernel = t.Kp == 64 ? gram_tc_kernel<true> : gram_tc_kernel<false>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
             return GAF_ERR_CUDA;
-        gram_tc_kernel<<<a.slices, kTcThreads, dyn, st>>>(t);
+        kernel<<<a.slices, t.Kp == 64 ? kTcThreadsWide : kTcThreads, dyn, st>>>(t);
         ++g_launches;
     } else {
         // CUDA cores, every gradient read once: one warp per tile pair, panels of D through shared memory
@@ -719,10 +720,16 @@ int gaf_stream_push(const void *g, int t, int64_t D, int dtype, double tau, floa
     const int grid = stream_grid(D, kStreamThreads, di.sms);
     if (dtype == GAF_F32) {
         stream_test_kernel<float><<<grid, kStreamThreads, 0, st>>>(a);
-        stream_add_kernel<float><<<grid, kStreamThreads, 0, st>>>(a);
+        if (launch_dependent(stream_add_kernel<float>, grid, kStreamThreads, st, a) != cudaSuccess) {
+            cudaGetLastError();
+            return GAF_ERR_CUDA;
+        }
     } else {
         stream_test_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, st>>>(a);
-        stream_add_kernel<__nv_bfloat16><<<grid, kStreamThreads, 0, st>>>(a);
+        if (launch_dependent(stream_add_kernel<__nv_bfloat16>, grid, kStreamThreads, st, a) != cudaSuccess) {
+            cudaGetLastError();
+            return GAF_ERR_CUDA;
+        }
     }
     g_launches += 2;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;

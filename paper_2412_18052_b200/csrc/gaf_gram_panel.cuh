@@ -1,7 +1,7 @@
 // Gram matrix G = X X^T for any number of gradients up to GAF_MAX_K and both input types, on
 // CUDA cores, reading every gradient ONCE from HBM (the general path: binary32 with more than 8
-// gradients, bfloat16 with more than 32; fewer go to the one-pass register-tiled kernel, bfloat16
-// up to 32 to the tensor cores).
+// gradients; fewer go to the one-pass register-tiled kernel, bfloat16 with 9 to 64 to the tensor
+// cores).
 //
 // The K x K matrix is cut into 8 x 8 tiles of pairs (upper triangle: P = T(T+1)/2 tile pairs for
 // T = ceil(K/8)).  One CTA per SM streams panels of the D axis -- all K rows x one chunk of

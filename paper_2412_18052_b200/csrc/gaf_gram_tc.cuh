@@ -1,4 +1,4 @@
-// Tensor-core Gram matrix for bfloat16 micro-gradients (K <= 32): G = X X^T with the
+// Tensor-core Gram matrix for bfloat16 micro-gradients (K <= 64): G = X X^T with the
 // D parameters as the contraction axis, on the 5th-generation tensor cores
 // (tcgen05.mma, accumulators in tensor memory).
 //
@@ -8,7 +8,7 @@
 //
 // Shape of one MMA: the K gradients are too few to fill the 128 rows of a tile, so R =
 // 128 / Kp different 64-element chunks of the D axis are stacked in the rows (Kp = K
-// rounded up to 8, 16 or 32): row c*Kp + i holds 64 consecutive elements of gradient i
+// rounded up to 8, 16, 32 or 64): row c*Kp + i holds 64 consecutive elements of gradient i
 // taken from chunk c.  The same shared-memory tile serves as both operands (A = B, both
 // K-major, 128-byte swizzle), so D = A A^T is 128 x 128 and its R diagonal Kp x Kp blocks
 // are R partial Gram matrices; the off-diagonal blocks mix different chunks and are
@@ -45,12 +45,13 @@ constexpr int kTcLoaderWarps = GAF_TC_LOADER_WARPS;
 constexpr int kTcLoaders = kTcLoaderWarps * 32;
 constexpr int kTcMmaWarp = 4 + kTcLoaderWarps;  // warps 0-3 epilogue, then the loaders, then the MMA issuer
 constexpr int kTcThreads = (kTcMmaWarp + 1) * 32;
+constexpr int kTcThreadsWide = kTcThreads + 128;  // 33..64 gradients: four more epilogue warps after the MMA warp
 constexpr int kTcStages = GAF_TC_STAGES;
 constexpr int kTcSub = GAF_TC_SUB;              // 128-row x 128-byte swizzle blocks per tile (one handshake per tile)
 constexpr int kTcBlockBytes = 128 * 128;        // one such block: 128 rows x 128 bytes
 constexpr int kTcStageBytes = kTcSub * kTcBlockBytes;
 constexpr int kTcDrain = 8 / kTcSub;            // tiles accumulated in tensor memory between drains (32 MMAs)
-constexpr int kTcMaxK = 32;
+constexpr int kTcMaxK = 64;
 constexpr int kTcTmemCols = 256;                // two accumulator buffers of 128 columns
 constexpr unsigned int kTcSpinLimit = 1u << 19;       // attempts of up to ~2 us each
 constexpr int kStatusTimeoutBit = 4;            // GAF_STATUS_TIMEOUT
@@ -58,7 +59,7 @@ constexpr int kStatusTimeoutBit = 4;            // GAF_STATUS_TIMEOUT
 struct GramTcArgs {
     const void *g[kTcMaxK];
     int K;                  // gradients
-    int Kp;                 // 8, 16 or 32
+    int Kp;                 // 8, 16, 32 or 64
     int64_t D;
     double *partials;       // [tile pair][slice][64]
     int tiles;              // ceil(K / 8)
@@ -175,7 +176,12 @@ struct GramTcShared {
     volatile int abort_flag;
 };
 
-__global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcArgs a) {
+// WIDE: Kp = 64.  A row's diagonal block is then 64 columns wide, twice what one epilogue thread can
+// carry in binary64 registers, so a second set of four epilogue warps (after the MMA warp; a warp reads
+// the tensor-memory lanes 32 (warp mod 4) .. + 31) takes the upper 32 columns of each block.
+template <bool WIDE>
+__global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcArgs a) {
+    constexpr int kThreads = WIDE ? kTcThreadsWide : kTcThreads;
     extern __shared__ unsigned char tc_dyn_smem[];
     __shared__ GramTcShared sh;
 
@@ -202,7 +208,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
         }
         for (int b = 0; b < 2; ++b) {
             tc_mbar_init(&sh.acc_full[b], 1);
-            tc_mbar_init(&sh.acc_empty[b], 128);         // every epilogue thread arrives
+            tc_mbar_init(&sh.acc_empty[b], WIDE ? 256 : 128);    // every epilogue thread arrives
         }
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -210,7 +216,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     }
     // rows of absent gradients (K < Kp) stay zero for the whole kernel
     if (K < Kp) {
-        for (int idx = threadIdx.x; idx < kTcStages * kTcSub * 128 * 8; idx += kTcThreads) {
+        for (int idx = threadIdx.x; idx < kTcStages * kTcSub * 128 * 8; idx += kThreads) {
             const int row = (idx >> 3) & 127;
             if ((row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
         }
@@ -227,6 +233,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     tc_fence_after_sync();
     const uint32_t tmem_base = sh.tmem_base;
 
+    // epilogue warps: which 32 rows (tensor-memory lanes) and which 32 columns of them this warp reads --
+    // the columns that hold the rows' diagonal block(s): the 32 on the diagonal, or one half of the 64
+    const int epi_q = warp & 3;
+    const int epi_col0 = WIDE ? (epi_q >> 1) * 64 + (warp > kTcMmaWarp ? 32 : 0) : epi_q * 32;
     double gsum[32];                                     // epilogue: this row's 32 loaded columns
 #pragma unroll
     for (int j = 0; j < 32; ++j) gsum[j] = 0.0;
@@ -321,7 +331,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
             if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag)) break;
             tc_fence_after_sync();
             uint32_t r[32];
-            tc_tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 128 + warp * 32), r);
+            tc_tmem_ld32(tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128 + epi_col0), r);
             tc_fence_before_sync();
             tc_mbar_arrive(&sh.acc_empty[buf]);
 #pragma unroll
@@ -343,12 +353,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     // the streaming part of this CTA is over: the finishing kernel, launched as a programmatic
     // dependent, may be placed now; it still waits for this whole grid before it reads the partials
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles <= 32 KB)
+    // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles <= 64 KB)
     double *red = reinterpret_cast<double *>(tiles);
-    if (warp < 4) {
-        const int row = warp * 32 + lane;                // row of the 128 x 128 result
+    if (warp < 4 || warp > kTcMmaWarp) {
+        const int row = epi_q * 32 + lane;               // row of the 128 x 128 result
         const int c = row / Kp, i = row % Kp;
-        const int off = c * Kp - warp * 32;              // where this chunk's block starts in the loaded columns
+        const int off = c * Kp - epi_col0;               // where this chunk's block starts in the loaded columns
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
             const int jj = j - off;
@@ -357,7 +367,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gram_tc_kernel(const __grid_con
     }
     __syncthreads();
     const int slices = gridDim.x;
-    for (int e = threadIdx.x; e < Kp * Kp; e += kTcThreads) {
+    for (int e = threadIdx.x; e < Kp * Kp; e += kThreads) {
         const int i = e / Kp, j = e % Kp;
         if (i > j || j >= K) continue;
         double s = 0.0;

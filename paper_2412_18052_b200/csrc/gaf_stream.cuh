@@ -49,6 +49,8 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_test_kernel(StreamAr
         s.na += (double)(v * v);
         s.ng += (double)(x * x);
     }
+    // the streaming part of this CTA is over: the add launch may start placing blocks
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     Sums3 blk = block_reduce(s, scratch);
     if (threadIdx.x == 0) {
         a.partials[3 * blockIdx.x] = blk.p;
@@ -80,6 +82,9 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_test_kernel(StreamAr
 // g <- g + g_i if step t was accepted.
 template <typename T>
 __global__ void __launch_bounds__(kStreamThreads, 2) stream_add_kernel(StreamArgs a) {
+    // launched as a programmatic dependent of the test: placed while that grid winds down, it waits
+    // here until the test has completed and its decision is visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (*reinterpret_cast<volatile int *>(&a.ctl->decision[a.t]) == 0) return;
     const T *g = static_cast<const T *>(a.g);
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

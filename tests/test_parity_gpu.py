@@ -161,9 +161,9 @@ def test_filter_maximum_k(ws, schedule):
     assert 1 < r["count"] < K
 
 
-@pytest.mark.parametrize("K", [9, 16, 24, 32])
+@pytest.mark.parametrize("K", [9, 16, 24, 32, 33, 48, 64])
 def test_filter_gram_first_on_tensor_cores(ws, K):
-    """bf16 with 9..32 gradients: the Gram matrix comes from the tcgen05 kernel."""
+    """bf16 with 9..64 gradients: the Gram matrix comes from the tcgen05 kernel."""
     w = _mix(K, 1_000_003 + 64 * K, "bf16", seed=200 + K)
     r = check_filter(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM)
     assert 1 < r["count"] < K
@@ -423,7 +423,7 @@ def test_auto_schedule_choice(ws):
              (8, 100_000, "bf16", gaf.GAF_SCHED_GRAM_FUSED), (6, 50_000, "bf16", gaf.GAF_SCHED_GRAM_FUSED),
              (9, 50_000, "f32", gaf.GAF_SCHED_GRAM), (32, 20_000, "f32", gaf.GAF_SCHED_GRAM),
              (33, 20_000, "f32", gaf.GAF_SCHED_STEPWISE), (16, 50_000, "bf16", gaf.GAF_SCHED_GRAM),
-             (33, 20_000, "bf16", gaf.GAF_SCHED_STEPWISE)]
+             (33, 20_000, "bf16", gaf.GAF_SCHED_GRAM), (64, 20_000, "bf16", gaf.GAF_SCHED_GRAM)]
     for K, D, dtype, want in cases:
         w = _mix(K, D, dtype, seed=11)
         gaf.gaf_filter_accumulate(w.grads, 0.97, ws)
