@@ -140,6 +140,8 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         const int threads = 32 * pa.pairs_per_cta * wpp;
         const int row_bytes = 16 << shift;
         const int dyn = kPanelStages * a.tiles * 8 * row_bytes;
+        // (bfloat16 comes here with a single gradient only: 2 to 8 take the register-tiled kernel, up to 64
+        // the tensor cores)
         void (*kernel)(GramPanelArgs) = nullptr;
         if (dtype == GAF_F32)
             kernel = shift == 7 ? gram_panel_kernel<float, 7, 4>

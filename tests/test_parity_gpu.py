@@ -409,8 +409,9 @@ def test_pairwise_small(ws, dtype):
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("K", [10, 16, 24, 32, 40, 48, 64])
 def test_pairwise_general_kernel_shapes(ws, dtype, K):
-    """The general CUDA-core Gram kernel in each of its shapes (warps sharing a tile pair, one warp
-    per pair, tile pairs split over groups of CTAs): several panels per CTA and a ragged last one."""
+    """More than 8 gradients: the general CUDA-core Gram kernel (binary32) in each of its shapes (warps
+    sharing a tile pair, one warp per pair, tile pairs split over groups of CTAs) and the tensor-core
+    kernel (bfloat16) in its 16-, 32- and 64-row forms: several panels or tiles per CTA, a ragged end."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     for D in (sms * 512 * 3 + 1234 + 3, 100_001):
         w = _mix(K, D, dtype, seed=300 + K)
