@@ -647,7 +647,8 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
     double *partials = reinterpret_cast<double *>(base + kExtraOffset);
     unsigned long long *bits = reinterpret_cast<unsigned long long *>(
         base + kExtraOffset + size_t(kBkMaxCtas + kBkMaxBuckets) * 64 * sizeof(double));
-    int grid = di.sms * 2;
+    // one wave: as many CTAs as are resident at once (two per SM up to 4 gradients, one beyond: registers)
+    int grid = di.sms * (K <= 4 ? 2 : 1);
     if (grid > kBkMaxCtas) grid = kBkMaxCtas;
     const int64_t n_oct = D / kOct;
     if (n_oct < grid) grid = n_oct > 0 ? int(n_oct) : 1;
@@ -655,6 +656,9 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
     BucketGramArgs ga{};
     for (int t = 0; t < K; ++t) ga.g[t] = grads[ord[t]];
     ga.D = D; ga.partials = partials; ga.ctl = reinterpret_cast<Control *>(base);
+    // the end of every CTA's range, kKeepL2Pct of L2 in all, is asked to stay in L2 for the mean pass
+    ga.keep_elems = int64_t(di.l2_bytes) * kKeepL2Pct / 100 / (int64_t(K) * int64_t(elem_bytes(dtype))) / grid;
+    ga.keep_elems = (ga.keep_elems + 7) / 8 * 8;
     int rc = dtype == GAF_F32 ? launch_bucket_gram<float>(ga, bt, K, grid, st)
                               : launch_bucket_gram<__nv_bfloat16>(ga, bt, K, grid, st);
     if (rc != GAF_OK) return rc;
@@ -664,14 +668,35 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
     wa.K = K; wa.D = D; wa.ctas = grid; wa.tau = tau; wa.partials = partials; wa.mask_out = mask_out;
     wa.dist_out = dist_out; wa.count_out = count_out; wa.bits = bits; wa.ctl = ga.ctl;
     for (int t = 0; t < K; ++t) wa.idx[t] = ord[t];
-    bucket_walk_kernel<<<S, 64 * kWalkChains, 0, st>>>(wa, bt);
+    {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(S); cfg.blockDim = dim3(64 * kWalkChains); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, bucket_walk_kernel, wa, bt) != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+    }
     ++g_launches;
 
     BucketMeanArgs ma{};
     for (int t = 0; t < K; ++t) ma.g[t] = grads[ord[t]];
     ma.K = K; ma.D = D; ma.out = macro_out; ma.bits = bits;
-    if (dtype == GAF_F32) bucket_mean_kernel<float><<<grid, kBkThreads, 0, st>>>(ma, bt);
-    else bucket_mean_kernel<__nv_bfloat16><<<grid, kBkThreads, 0, st>>>(ma, bt);
+    {
+        cudaLaunchConfig_t cfg{};
+        // (its own grid, two CTAs per SM: the ranges need not be those of the Gram pass)
+        int mean_grid = di.sms * 2;
+        if (mean_grid > kBkMaxCtas) mean_grid = kBkMaxCtas;
+        if (n_oct < mean_grid) mean_grid = n_oct > 0 ? int(n_oct) : 1;
+        cfg.gridDim = dim3(mean_grid); cfg.blockDim = dim3(kBkThreads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const cudaError_t err = dtype == GAF_F32 ? cudaLaunchKernelEx(&cfg, bucket_mean_kernel<float>, ma, bt)
+                                                 : cudaLaunchKernelEx(&cfg, bucket_mean_kernel<__nv_bfloat16>, ma, bt);
+        if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+    }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }

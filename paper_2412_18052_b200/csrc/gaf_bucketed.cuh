@@ -44,12 +44,13 @@ __device__ __forceinline__ void cta_range(int64_t D, int c, int G, int64_t &lo, 
 struct BucketGramArgs {
     const void *g[kGsMaxK];                 // processing order
     int64_t D;
+    int64_t keep_elems;                     // the last so many elements of every CTA's range are loaded "keep in L2"
     double *partials;                       // [slot][64], slot = cta + bucket
     Control *ctl;
 };
 
 template <typename T, int KT>
-__global__ void __launch_bounds__(kBkThreads, 1)
+__global__ void __launch_bounds__(kBkThreads, (KT <= 4 ? 2 : 1))
 bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_constant__ BucketTable bt) {
     constexpr int NP = KT * (KT + 1) / 2;
     constexpr int N = GsVec<T>::N;
@@ -58,7 +59,8 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
     const T *row[KT];
 #pragma unroll
     for (int r = 0; r < KT; ++r) row[r] = static_cast<const T *>(a.g[r]);
-    const uint64_t pol = l2_policy_evict_first();
+    // the mean pass walks every CTA's range from its end: the end of the range is asked to stay in L2
+    const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
     if (blockIdx.x == 0 && threadIdx.x == 0) a.ctl->status = 0;     // first kernel of the operation
 
     int64_t lo, hi;
@@ -92,6 +94,8 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
                 const int64_t q = qw + lane;
                 if (q < n_vec) {
                     float x[KT][N];
+#pragma unroll
+                    const uint64_t pol = (s0 + q * N >= hi - a.keep_elems) ? pol_last : pol_first;
 #pragma unroll
                     for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], s0 + q * N, pol, x[r]);
                     int p = 0;
@@ -130,6 +134,8 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
         if (bt.off[b + 1] >= hi || b + 1 >= bt.S) break;
         ++b;
     }
+    // the per-bucket walk is launched as a programmatic dependent: its blocks may be placed now
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 struct BucketWalkArgs {
@@ -176,6 +182,10 @@ bucket_walk_kernel(const __grid_constant__ BucketWalkArgs a, const __grid_consta
         c_last = lo;
     }
     const int p = threadIdx.x & 63, chain = threadIdx.x >> 6;
+    // programmatic dependent of the Gram pass: wait for that grid and its partial sums; the mean pass
+    // behind this kernel may be placed at once (it waits for this grid in turn)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     {
         const int n = c_last - c_first + 1;
         const int per = (n + kWalkChains - 1) / kWalkChains;
@@ -243,8 +253,12 @@ bucket_mean_kernel(const __grid_constant__ BucketMeanArgs a, const __grid_consta
     __shared__ int n_list;
     int64_t lo, hi;
     cta_range(a.D, blockIdx.x, gridDim.x, lo, hi);
+    // programmatic dependent of the per-bucket walk: wait for its accept bits
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (lo >= hi) return;
-    int b = bucket_of(bt, lo);
+    // the range is walked from its END (buckets last to first, each from its end): the Gram pass
+    // walked it from the start, so its last-read lines are the ones still in L2
+    int b = bucket_of(bt, hi - 1);
     while (true) {
         const int64_t s0 = lo > bt.off[b] ? lo : bt.off[b];
         const int64_t s1 = hi < bt.off[b + 1] ? hi : bt.off[b + 1];
@@ -262,7 +276,7 @@ bucket_mean_kernel(const __grid_constant__ BucketMeanArgs a, const __grid_consta
             const float cdiv = (float)n;
             const int64_t n_oct = (s1 - s0) / kOct;
             for (int64_t o = threadIdx.x; o < n_oct; o += kBkThreads) {
-                const int64_t e = s0 + o * kOct;
+                const int64_t e = s0 + (n_oct - 1 - o) * kOct;
                 float v[8];
                 RawOct<T>::load(list[0], e).widen(v);
                 for (int i = 1; i < n; i += 3) {
@@ -291,8 +305,8 @@ bucket_mean_kernel(const __grid_constant__ BucketMeanArgs a, const __grid_consta
                 a.out[e] = v / cdiv;
             }
         }
-        if (bt.off[b + 1] >= hi || b + 1 >= bt.S) break;
-        ++b;
+        if (bt.off[b] <= lo || b == 0) break;
+        --b;
     }
 }
 
