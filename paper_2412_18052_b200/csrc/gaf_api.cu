@@ -211,7 +211,8 @@ int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
 // One-launch form of the Gram-first schedule (gaf_fused.cuh).  Returns GAF_OK when it was
 // launched, GAF_ERR_UNSUPPORTED when this device or K does not allow it, or an error code.
 constexpr int kKeepL2Pct = 10;          // share of L2 the Gram pass asks to keep for the second pass
-                                        // (measured: larger shares slow both passes down)
+                                        // ("evict last" lines live in the persisting part of L2, 24.9 MB by
+                                        // default on this GPU; larger shares slow both passes down)
 // Shared memory of one SM given to parked rounds.  The rest of the L1/shared array stays L1, which the
 // loads in flight need: beyond about 60 % shared memory both passes lose more than parking gains.
 constexpr int kParkBytesPerSm = 128 << 10;
