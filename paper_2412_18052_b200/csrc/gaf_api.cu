@@ -49,6 +49,42 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline size_t elem_bytes(int dtype) { return dtype == GAF_F32 ? 4 : 2; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Launch `kernel` as a programmatic dependent of the launch before it on the stream: its blocks may be
+// placed while that grid winds down; the kernel itself waits (griddepcontrol.wait) for that grid.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int threads, cudaStream_t st, const Args &...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// macro_out (D floats) must not overlap any input gradient.
+bool overlaps_inputs(const float *macro_out, const void *const *grads, int K, int64_t D, int dtype) {
+    const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
+    for (int i = 0; i < K; ++i) {
+        const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
+        const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
+        if (o0 < g1 && g0 < o1) return true;
+    }
+    return false;
+}
+
+// `order` (NULL = identity) must be a permutation of 0..K-1; copies it to `ord`.
+bool read_order(const int32_t *order, int K, int32_t *ord) {
+    bool seen[GAF_MAX_K] = {false};
+    for (int t = 0; t < K; ++t) {
+        const int32_t i = order ? order[t] : t;
+        if (i < 0 || i >= K || seen[i]) return false;
+        seen[i] = true;
+        ord[t] = i;
+    }
+    return true;
+}
+
 // CTAs for a streaming kernel of `threads` threads that handles 8 elements per
 // thread and iteration: two per SM, fewer when D is small.
 int stream_grid(int64_t D, int threads, int sms) {
@@ -163,14 +199,8 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         ++g_launches;
     }
     {
-        // programmatic dependent launch: the finishing blocks are placed while the Gram kernel winds down
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(pairs); cfg.blockDim = dim3(64 * kFinishParts); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        const cudaError_t err = cudaLaunchKernelEx(&cfg, gram_finish_kernel, a);
+        // the finishing blocks are placed while the Gram kernel winds down
+        const cudaError_t err = launch_dependent(gram_finish_kernel, pairs, 64 * kFinishParts, st, a);
         ++g_launches;
         if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     }
@@ -337,15 +367,8 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     for (int t = 0; t < K; ++t) m.g[t] = g[ord[t]];
     m.K = K; m.D = D; m.out = macro_out; m.ctl = ctl;
     const int grid = stream_grid(D, kMsThreads, sms);
-    // programmatic dependent launch: the blocks may be placed while the Gram pass winds down
-    // (its last CTA is still totalling partials); the kernel itself waits for that grid
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kMsThreads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, masked_mean_kernel<T>, m);
+    // the blocks may be placed while the Gram pass winds down (its last CTA is still totalling partials)
+    const cudaError_t err = launch_dependent(masked_mean_kernel<T>, grid, kMsThreads, st, m);
     ++g_launches;
     if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
@@ -360,19 +383,6 @@ bool auto_one_launch(int K, int64_t D, int dtype, const DeviceInfo &di) {
 int check_workspace(const void *ws, size_t have, size_t need) {
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || have < need) return GAF_ERR_WORKSPACE;
     return GAF_OK;
-}
-
-// Launch `kernel` as a programmatic dependent of the launch before it on the stream: its blocks may be
-// placed while that grid winds down; the kernel itself waits (griddepcontrol.wait) for that grid.
-template <typename Args>
-cudaError_t launch_dependent(void (*kernel)(Args), int grid, int threads, cudaStream_t st, const Args &args) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args);
 }
 
 template <typename T>
@@ -508,23 +518,8 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     if (tau != tau) return GAF_ERR_ARG;
     if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
     int32_t ord[GAF_MAX_K];
-    {
-        bool seen[GAF_MAX_K] = {false};
-        for (int t = 0; t < K; ++t) {
-            int32_t i = order ? order[t] : t;
-            if (i < 0 || i >= K || seen[i]) return GAF_ERR_ARG;
-            seen[i] = true;
-            ord[t] = i;
-        }
-    }
-    {
-        const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
-        for (int i = 0; i < K; ++i) {
-            const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
-            const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
-            if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
-        }
-    }
+    if (!read_order(order, K, ord)) return GAF_ERR_ARG;
+    if (overlaps_inputs(macro_out, grads, K, D, dtype)) return GAF_ERR_ALIAS;
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
     DeviceInfo di;
     if (!device_info(&di)) return GAF_ERR_CUDA;
@@ -570,14 +565,7 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
     if ((!macro_out && D > 0) || !mask_out || !count_out || !seed_out) return GAF_ERR_ARG;
     if (tau != tau) return GAF_ERR_ARG;
     if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
-    {
-        const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
-        for (int i = 0; i < K; ++i) {
-            const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
-            const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
-            if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
-        }
-    }
+    if (overlaps_inputs(macro_out, grads, K, D, dtype)) return GAF_ERR_ALIAS;
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K))) return rc;
     DeviceInfo di;
     if (!device_info(&di)) return GAF_ERR_CUDA;
@@ -619,23 +607,8 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
     }
     if (!aligned16(macro_out)) return GAF_ERR_ALIGN;
     int32_t ord[GAF_MAX_K];
-    {
-        bool seen[GAF_MAX_K] = {false};
-        for (int t = 0; t < K; ++t) {
-            const int32_t i = order ? order[t] : t;
-            if (i < 0 || i >= K || seen[i]) return GAF_ERR_ARG;
-            seen[i] = true;
-            ord[t] = i;
-        }
-    }
-    {
-        const uintptr_t o0 = reinterpret_cast<uintptr_t>(macro_out), o1 = o0 + size_t(D) * 4;
-        for (int i = 0; i < K; ++i) {
-            const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads[i]);
-            const uintptr_t g1 = g0 + size_t(D) * elem_bytes(dtype);
-            if (o0 < g1 && g0 < o1) return GAF_ERR_ALIAS;
-        }
-    }
+    if (!read_order(order, K, ord)) return GAF_ERR_ARG;
+    if (overlaps_inputs(macro_out, grads, K, D, dtype)) return GAF_ERR_ALIAS;
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + bucketed_extra_bytes())) return rc;
     DeviceInfo di;
     if (!device_info(&di)) return GAF_ERR_CUDA;
@@ -669,14 +642,9 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
     wa.K = K; wa.D = D; wa.ctas = grid; wa.tau = tau; wa.partials = partials; wa.mask_out = mask_out;
     wa.dist_out = dist_out; wa.count_out = count_out; wa.bits = bits; wa.ctl = ga.ctl;
     for (int t = 0; t < K; ++t) wa.idx[t] = ord[t];
-    {
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(S); cfg.blockDim = dim3(64 * kWalkChains); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, bucket_walk_kernel, wa, bt) != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+    if (launch_dependent(bucket_walk_kernel, S, 64 * kWalkChains, st, wa, bt) != cudaSuccess) {
+        cudaGetLastError();
+        return GAF_ERR_CUDA;
     }
     ++g_launches;
 
@@ -684,18 +652,13 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
     for (int t = 0; t < K; ++t) ma.g[t] = grads[ord[t]];
     ma.K = K; ma.D = D; ma.out = macro_out; ma.bits = bits;
     {
-        cudaLaunchConfig_t cfg{};
         // (its own grid, two CTAs per SM: the ranges need not be those of the Gram pass)
         int mean_grid = di.sms * 2;
         if (mean_grid > kBkMaxCtas) mean_grid = kBkMaxCtas;
         if (n_oct < mean_grid) mean_grid = n_oct > 0 ? int(n_oct) : 1;
-        cfg.gridDim = dim3(mean_grid); cfg.blockDim = dim3(kBkThreads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        const cudaError_t err = dtype == GAF_F32 ? cudaLaunchKernelEx(&cfg, bucket_mean_kernel<float>, ma, bt)
-                                                 : cudaLaunchKernelEx(&cfg, bucket_mean_kernel<__nv_bfloat16>, ma, bt);
+        const cudaError_t err = dtype == GAF_F32
+            ? launch_dependent(bucket_mean_kernel<float>, mean_grid, kBkThreads, st, ma, bt)
+            : launch_dependent(bucket_mean_kernel<__nv_bfloat16>, mean_grid, kBkThreads, st, ma, bt);
         if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     }
     ++g_launches;
