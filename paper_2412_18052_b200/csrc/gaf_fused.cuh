@@ -3,17 +3,18 @@
 // The two-launch form (gaf_gramfilter.cuh) reads every gradient once for the Gram
 // matrix and the accepted ones a second time for g/c (Eq. 5).  When the whole call
 // lasts tens of microseconds, what the second pass has to fetch again is a large part
-// of the cost.  Here one co-resident grid does both passes, so that what a thread
-// loaded last in the first pass is still ON CHIP when the second pass starts:
+// of the cost.  Here one co-resident grid does both passes, so that part of what the
+// first pass read is still ON CHIP when the second pass starts:
 //   pass 1   every thread walks its vectors (grid-stride), accumulating the Gram
 //            partial sums exactly as gram_small_kernel does, and parks the raw loads
-//            of its last R rounds in shared memory;
+//            of its FIRST R rounds in shared memory (the last rounds are the ones L2
+//            still holds afterwards: shared memory and L2 then keep different data);
 //   decide   per-CTA partials, last CTA to arrive totals them in fixed order, walks
 //            Algorithm 1 (Eq. 4 in binary64) on the Gram matrix and publishes the accept
-//            bits; the other CTAs wait for it (bounded spin on a generation word);
-//   pass 2   the same thread visits the same vectors: the parked rounds straight from
-//            shared memory, then the rest from the end towards the start (the rounds
-//            just before the parked ones were loaded "keep in L2"), adding the accepted
+//            bits in one polled word; the other CTAs wait for it (bounded spin);
+//   pass 2   the same thread visits the same vectors: the rounds that were not parked
+//            from the last one down (the end of the vectors was loaded "keep in L2"),
+//            then the parked rounds straight from shared memory, adding the accepted
 //            gradients in processing order in binary32 and dividing by c.
 // Same sums, same order of additions as the two-launch form: identical outputs.
 // The grid must be co-resident (cooperative launch); every wait is bounded and ends in
@@ -126,7 +127,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     };
 
     const int64_t tail0 = n_vec * N;
-    // ---- pass 1: Gram partial sums; the last rounds stay in shared memory ----
+    // ---- pass 1: Gram partial sums; the first rounds stay in shared memory ----
     int since_flush = 0;
     for (int64_t j = 0; j < rounds; ++j) {
         const int64_t q = warp_first + j * stride + lane;
