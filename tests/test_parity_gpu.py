@@ -233,6 +233,40 @@ def test_filter_random_cases(ws):
         check_filter(w.grads, tau, ws, order=order, schedule=schedule, expect_status=None)
 
 
+def test_random_cases_all_entry_points(ws):
+    """A seeded sweep over every Gram path and schedule: 1..64 gradients, lengths from 0 to a few
+    waves with ragged ends, both types, all schedules, filter / pairwise matrix / any-seed variant.
+    (Thresholds above 1 are only drawn for vectors long enough not to cancel: see the tolerance notes.)"""
+    rng = np.random.RandomState(77)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for case in range(240):
+        K = int(rng.choice([1, 2, 3, 4, 5, 6, 7, 8, 9, 12, 16, 17, 24, 31, 32, 33, 40, 41, 48, 57, 64]))
+        if rng.rand() < 0.3:
+            D = int(rng.randint(100_000, 1_500_000))
+        else:
+            D = int(rng.choice([0, 1, 2, 3, 5, 8, 17, 100, 511, 512, 513, 4096, 65_537]))
+        if rng.rand() < 0.15:
+            D = int(sms * 512 * rng.randint(1, 4) * (4 if rng.rand() < 0.5 else 8) + rng.randint(-9, 9))
+        if K > 16:
+            D = min(D, 300_000)
+        dtype = "bf16" if rng.rand() < 0.5 else "f32"
+        tau = float(rng.choice([0.3, 0.8, 0.97, 1.0, 1.05, 1.6, 2.0, -1.0]))
+        if D < 2000 and tau > 1.0:
+            tau = 1.0
+        order = [int(x) for x in rng.permutation(K)] if rng.rand() < 0.5 else None
+        schedule = int(rng.choice([0, 1, 2] + ([3] if 2 <= K <= 8 else [])))
+        rho = rng.uniform(-0.6, 0.95, size=K)
+        w = workloads.mixture(K, D, dtype, list(rho), int(rng.randint(1 << 30)), device="cuda",
+                              sigma=float(rng.choice([1e-3, 1.0, 30.0])))
+        kind = rng.rand()
+        if kind < 0.6:
+            check_filter(w.grads, tau, ws, order=order, schedule=schedule, expect_status=None)
+        elif kind < 0.85:
+            check_pairwise(w.grads, ws)
+        else:
+            check_any_seed(w.grads, tau, ws)
+
+
 @pytest.mark.parametrize("dtype", DTYPES)
 def test_gram_loop_ends_inside_a_warp_at_the_flush_period(ws, dtype):
     """Lengths for which some lanes of a warp run exactly 16 rounds of the Gram loop (one
