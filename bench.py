@@ -509,7 +509,7 @@ def run_ours(args):
             },
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak,
+                "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0,
                 "traffic": (ncu_traffic_config2(masks, n_sets, steps)
                             if (cfg == 2 and sched_used == 3 and abs(args.tau - 0.97) < 1e-12) else None),
                 "peak_kind": f"of {peak_kind}",
