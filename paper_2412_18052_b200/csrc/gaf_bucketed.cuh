@@ -73,17 +73,18 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
         if (s1 > s0) {
             for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
             __syncwarp();
-            float acc[NP];
+            using Acc = typename GsAcc<T, KT>::type;
+            Acc acc[NP];
 #pragma unroll
-            for (int p = 0; p < NP; ++p) acc[p] = 0.0f;
+            for (int p = 0; p < NP; ++p) acc[p] = Acc(0);
             auto flush = [&]() {
 #pragma unroll
                 for (int p = 0; p < NP; ++p) {
-                    float v = acc[p];
+                    Acc v = acc[p];
 #pragma unroll
                     for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
                     if (lane == 0) sacc[warp][p] += (double)v;
-                    acc[p] = 0.0f;
+                    acc[p] = Acc(0);
                 }
             };
             // s0 is a multiple of 8 elements (bucket offsets and CTA ranges are), so vector loads are aligned
@@ -103,13 +104,13 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
                     for (int r = 0; r < KT; ++r)
 #pragma unroll
                         for (int c = r; c < KT; ++c, ++p) {
-                            float s = acc[p];
+                            Acc s = acc[p];
 #pragma unroll
-                            for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
+                            for (int k = 0; k < N; ++k) s = gs_fma(x[r][k], x[c][k], s);
                             acc[p] = s;
                         }
                 }
-                if (++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+                if (GsAcc<T, KT>::kPeriodicFlush && ++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
             }
             const int64_t t0 = s0 + n_vec * N;          // fewer than N leftover elements
             if (t0 + threadIdx.x < s1) {
@@ -120,7 +121,7 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
 #pragma unroll
                 for (int r = 0; r < KT; ++r)
 #pragma unroll
-                    for (int c = r; c < KT; ++c, ++p) acc[p] = fmaf(x[r], x[c], acc[p]);
+                    for (int c = r; c < KT; ++c, ++p) acc[p] = gs_fma(x[r], x[c], acc[p]);
             }
             flush();
             __syncthreads();

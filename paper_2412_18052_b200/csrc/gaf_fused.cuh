@@ -112,17 +112,18 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     const int64_t warp_first = (int64_t)blockIdx.x * blockDim.x + (tid & ~31);
     const int64_t rounds = warp_first < n_vec ? (n_vec - warp_first + stride - 1) / stride : 0;
     const int64_t parked_rounds = rounds < a.park_rounds ? rounds : a.park_rounds;   // the FIRST ones
-    float acc[NP];
+    using Acc = typename GsAcc<T, KT>::type;
+    Acc acc[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) acc[p] = 0.0f;
+    for (int p = 0; p < NP; ++p) acc[p] = Acc(0);
     auto flush = [&]() {
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
-            float v = acc[p];
+            Acc v = acc[p];
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
             if (lane == 0) sacc[warp][p] += (double)v;
-            acc[p] = 0.0f;
+            acc[p] = Acc(0);
         }
     };
 
@@ -150,13 +151,13 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
             for (int r = 0; r < KT; ++r)
 #pragma unroll
                 for (int c = r; c < KT; ++c, ++p) {
-                    float s = acc[p];
+                    Acc s = acc[p];
 #pragma unroll
-                    for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
+                    for (int k = 0; k < N; ++k) s = gs_fma(x[r][k], x[c][k], s);
                     acc[p] = s;
                 }
         }
-        if (++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+        if (GsAcc<T, KT>::kPeriodicFlush && ++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
     }
     // ragged tail (D mod N elements), first CTA
     if (blockIdx.x == 0 && tail0 + tid < a.D) {
@@ -168,7 +169,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
 #pragma unroll
         for (int r = 0; r < KT; ++r)
 #pragma unroll
-            for (int c = r; c < KT; ++c, ++p) acc[p] = fmaf(x[r], x[c], acc[p]);
+            for (int c = r; c < KT; ++c, ++p) acc[p] = gs_fma(x[r], x[c], acc[p]);
     }
     flush();
     __syncthreads();

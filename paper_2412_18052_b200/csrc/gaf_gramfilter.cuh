@@ -339,8 +339,27 @@ __device__ __forceinline__ void total_gram_partials(const double *part, int n_ct
     }
 }
 
+// Accumulator of the register-tiled Gram kernels (K <= 8).
+// binary32 inputs, up to 4 gradients: binary64.  A product of two binary32 values is exact in binary64, so
+// the Gram sums are exact up to binary64 rounding and need no periodic flush; binary64 FMAs (half the
+// binary32 rate on this GPU) keep up with HBM here (measured: the same pass time, and a shorter call because
+// the flushes are gone).  With 5 to 8 gradients there are up to 1.4 binary64 operations per byte read and
+// the long passes, which run under the power cap, lost 8 %: binary32 chains there.
+// bfloat16 inputs: binary32 chains (a product of two bfloat16 values is exact in binary32; there are twice
+// as many products per byte), widened to binary64 every kGsFlushEvery rounds like the binary32 chains above.
+template <typename T, int KT> struct GsAcc {
+    using type = float;
+    static constexpr bool kPeriodicFlush = true;
+};
+template <> struct GsAcc<float, 1> { using type = double; static constexpr bool kPeriodicFlush = false; };
+template <> struct GsAcc<float, 2> { using type = double; static constexpr bool kPeriodicFlush = false; };
+template <> struct GsAcc<float, 3> { using type = double; static constexpr bool kPeriodicFlush = false; };
+template <> struct GsAcc<float, 4> { using type = double; static constexpr bool kPeriodicFlush = false; };
+__device__ __forceinline__ float gs_fma(float a, float b, float s) { return fmaf(a, b, s); }
+__device__ __forceinline__ double gs_fma(float a, float b, double s) { return fma((double)a, (double)b, s); }
+
 template <typename T, int KT>
-__global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_constant__ GramSmallArgs a) {
+__global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1)) gram_small_kernel(const __grid_constant__ GramSmallArgs a) {
     constexpr int NP = KT * (KT + 1) / 2;   // upper triangle
     constexpr int N = GsVec<T>::N;
     __shared__ double sacc[kGsThreads / 32][NP];
@@ -354,18 +373,19 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
 #pragma unroll
     for (int r = 0; r < KT; ++r) row[r] = static_cast<const T *>(a.g[r]);
 
-    float acc[NP];
+    using Acc = typename GsAcc<T, KT>::type;
+    Acc acc[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) acc[p] = 0.0f;
+    for (int p = 0; p < NP; ++p) acc[p] = Acc(0);
 
     auto flush = [&]() {
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
-            float v = acc[p];
+            Acc v = acc[p];
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
             if (lane == 0) sacc[warp][p] += (double)v;
-            acc[p] = 0.0f;
+            acc[p] = Acc(0);
         }
     };
 
@@ -391,13 +411,13 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
             for (int r = 0; r < KT; ++r)
 #pragma unroll
                 for (int c = r; c < KT; ++c, ++p) {
-                    float s = acc[p];
+                    Acc s = acc[p];
 #pragma unroll
-                    for (int k = 0; k < N; ++k) s = fmaf(x[r][k], x[c][k], s);
+                    for (int k = 0; k < N; ++k) s = gs_fma(x[r][k], x[c][k], s);
                     acc[p] = s;
                 }
         }
-        if (++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+        if (GsAcc<T, KT>::kPeriodicFlush && ++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
     }
     // ragged tail (D mod N elements), first CTA
     const int64_t tail0 = n_vec * N;
@@ -410,7 +430,7 @@ __global__ void __launch_bounds__(kGsThreads, 1) gram_small_kernel(const __grid_
 #pragma unroll
         for (int r = 0; r < KT; ++r)
 #pragma unroll
-            for (int c = r; c < KT; ++c, ++p) acc[p] = fmaf(x[r], x[c], acc[p]);
+            for (int c = r; c < KT; ++c, ++p) acc[p] = gs_fma(x[r], x[c], acc[p]);
     }
     flush();
     // the streaming part of this CTA is over: a kernel launched as a programmatic dependent
