@@ -22,11 +22,13 @@
  *   - Gradient buffers are read-only.  Every device pointer must be 16-byte
  *     aligned (else GAF_ERR_ALIGN).  D need not be a multiple of anything; with
  *     D == 0 the element buffers may be NULL.
- *   - dtype: GAF_F32 = IEEE binary32, GAF_BF16 = bfloat16.  All arithmetic on
- *     elements is binary32; sums are carried in binary64 from the thread level
- *     up and reduced in a fixed order, so results are bitwise reproducible on
- *     the same GPU model.  The scalar arithmetic of Eq. 4 and the comparison
- *     with tau are binary64.
+ *   - dtype: GAF_F32 = IEEE binary32, GAF_BF16 = bfloat16.  Arithmetic on
+ *     elements is binary32 (products of at most 64 pairs are summed in binary32
+ *     before they are widened; the Gram sums of up to 4 binary32 gradients are
+ *     taken in binary64 throughout, where every product is exact); sums are
+ *     carried in binary64 from the thread level up and reduced in a fixed
+ *     order, so results are bitwise reproducible on the same GPU model.  The
+ *     scalar arithmetic of Eq. 4 and the comparison with tau are binary64.
  *   - Conventions where the paper is silent: a pair with a zero-norm member has
  *     cos := 0 (distance 1); cos is clamped to [-1, 1]; a NaN distance is
  *     rejected.  Either event sets a bit in the status word (see
