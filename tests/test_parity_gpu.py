@@ -471,6 +471,18 @@ def test_auto_schedule_choice(ws):
     assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM
 
 
+def test_gram_sums_of_few_fp32_gradients_are_exact_to_binary64_rounding(ws):
+    """Up to 4 binary32 gradients the Gram kernels accumulate in binary64, where every product is exact:
+    the Gram matrix agrees with the oracle's to binary64 rounding, not merely to binary32 precision."""
+    from oracle import gaf_oracle as orc
+    for K in (2, 3, 4):
+        w = _mix(K, 1_000_003, "f32", seed=40 + K)
+        _, gram = gaf.gaf_pairwise_cosdist(w.grads, ws)
+        o_gram, _ = orc.pairwise_cosdist([workloads.as_numpy_bits(g) for g in w.grads])
+        nrm = np.sqrt(np.diag(o_gram))
+        assert float(np.max(np.abs(gram.cpu().numpy() - o_gram) / np.outer(nrm, nrm))) < 1e-12
+
+
 def test_pairwise_zero_norm_row(ws):
     w = _mix(4, 5001, "f32", seed=2)
     w.grads[2].zero_()
