@@ -72,7 +72,8 @@ enum {
                                    pays off (K <= 32; bfloat16: K <= 64), else stepwise.
                                    For K <= 8 the one-launch form is taken for binary32 inputs of
                                    at most 512 MB in all, and for bfloat16 inputs except 8
-                                   gradients of more than 1 GB in all (tensor-core Gram then). */
+                                   gradients of more than 1 GB in all (tensor-core Gram then);
+                                   if the device refuses the co-resident launch, two launches. */
     GAF_SCHED_STEPWISE = 1,     /* streaming: one launch per step; each launch adds the
                                    gradient accepted at step t to the running sum and, in
                                    the same pass, takes the three dot products of the

@@ -528,6 +528,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     double *partials = reinterpret_cast<double *>(base + kPartialsOffset);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
+    const bool library_choice = schedule == GAF_SCHED_AUTO;
     if (schedule == GAF_SCHED_AUTO) {
         // Gram-first moves fewer bytes whenever its one-pass Gram kernel applies
         const bool ws_ok = workspace_bytes >= kExtraOffset + pairwise_extra_bytes(K);
@@ -542,12 +543,22 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
     if (schedule == GAF_SCHED_GRAM || schedule == GAF_SCHED_GRAM_FUSED) {
         if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K)))
             return rc;
-        const bool one_launch = schedule == GAF_SCHED_GRAM_FUSED;
-        return dtype == GAF_F32
-            ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                       count_out, nullptr, base, di, one_launch, st)
-            : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                               count_out, nullptr, base, di, one_launch, st);
+        auto run = [&](bool one_launch) {
+            return dtype == GAF_F32
+                ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
+                                           count_out, nullptr, base, di, one_launch, st)
+                : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
+                                                   count_out, nullptr, base, di, one_launch, st);
+        };
+        int rc = run(schedule == GAF_SCHED_GRAM_FUSED);
+        if (rc != GAF_OK && library_choice && schedule == GAF_SCHED_GRAM_FUSED) {
+            // the co-resident launch was refused (for example the device cannot hold the whole grid right
+            // now): the library's own choice falls back to the two-launch form, an explicit request does not
+            g_launches = 0;
+            g_schedule = GAF_SCHED_GRAM;
+            rc = run(false);
+        }
+        return rc;
     }
     return dtype == GAF_F32
         ? launch_stepwise<float>(grads, K, D, tau, ord, macro_out, mask_out, dist_out, count_out,
@@ -585,11 +596,20 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
         if (rc != GAF_OK) return rc;
         return cudaMemsetAsync(seed_out, 0, sizeof(int32_t), st) == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
     }
-    return dtype == GAF_F32
-        ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out, count_out,
-                                   seed_out, base, di, auto_one_launch(K, D, dtype, di), st)
-        : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
-                                           count_out, seed_out, base, di, auto_one_launch(K, D, dtype, di), st);
+    auto run = [&](bool one_launch) {
+        return dtype == GAF_F32
+            ? launch_gram_first<float>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out, count_out,
+                                       seed_out, base, di, one_launch, st)
+            : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
+                                               count_out, seed_out, base, di, one_launch, st);
+    };
+    const bool one_launch = auto_one_launch(K, D, dtype, di);
+    int rc = run(one_launch);
+    if (rc != GAF_OK && one_launch) {       // co-resident launch refused: two launches
+        g_launches = 0;
+        rc = run(false);
+    }
+    return rc;
 }
 
 int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, int dtype, double tau,
