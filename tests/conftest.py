@@ -13,6 +13,14 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "slow: full-size workloads")
 
 
+def pytest_sessionstart(session):
+    """Compile the CUDA library if the tree does not hold it yet (a fresh checkout): nvcc works
+    without a GPU.  An existing library is used as it is."""
+    from paper_2412_18052_b200 import build as cuda_build
+    if not os.path.exists(cuda_build.LIB):
+        cuda_build.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
