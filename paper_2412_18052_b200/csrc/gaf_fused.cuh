@@ -26,7 +26,7 @@
 
 namespace gaf {
 
-constexpr unsigned int kFusedSpinLimit = 1u << 22;   // polls of >= 200 ns each: about a second
+constexpr unsigned int kFusedSpinLimit = 1u << 23;   // polls of an L2 round trip plus a 40 ns sleep each: seconds
 
 struct GramFusedArgs {
     const void *g[kGsMaxK];                 // processing order (original order in any-seed mode)
@@ -184,17 +184,21 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
         }
         a.partials[(size_t)tid * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     }
-    __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned int old = atomicInc(&ctl->ticket, gridDim.x - 1);
+        // Ticket with release and acquire semantics at GPU scope, in place of a fence by every thread plus a
+        // relaxed atomic: the partials written above happen before it through the barrier, so they are
+        // visible to whoever sees this ticket, and the last CTA's loads below, behind the next barrier, see
+        // every other CTA's partials.  (It wraps to 0 after the last ticket: the workspace is reusable.)
+        unsigned int old;
+        asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;"
+                     : "=r"(old) : "l"(&ctl->ticket), "r"(gridDim.x - 1) : "memory");
         is_last = (old == gridDim.x - 1);
     }
     __syncthreads();
 
     // ---- decide: last CTA totals the partials in fixed order and walks Algorithm 1 ----
     if (is_last) {
-        __threadfence();
         total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
         __syncthreads();
         // the accept bits go out first, in the polled word itself; the outputs follow
@@ -218,7 +222,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
         if (!is_last) {
             unsigned int polls = 0;
             while (((word = ld_relaxed_u32(&ctl->fused_word)) >> 16) == gen0) {
-                __nanosleep(200);
+                __nanosleep(40);
                 if (++polls > kFusedSpinLimit) { ok = false; break; }
             }
         }
