@@ -92,7 +92,7 @@ def gram_first_bytes(mask_in_order, K, D, b):
 NCU_TRAFFIC = {
     "sources": ["paper_2412_18052_b200/csrc/gaf_fused.cuh", "paper_2412_18052_b200/csrc/gaf_gramfilter.cuh",
                 "paper_2412_18052_b200/csrc/gaf_device.cuh"],
-    "sha256": "d95a50910f8d1a73134bc0cf82e2488d654d8bee0422490bb71cff52d9e94883",
+    "sha256": "20ad1f8887539529e153445b7125b860e388b39340d38eaa53b88b2474250306",
     "gram_fused_kernel<float,4>": {2: 233.5e6, 3: 261.6e6},
 }
 

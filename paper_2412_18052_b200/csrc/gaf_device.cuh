@@ -39,6 +39,20 @@ constexpr size_t kPartialsOffset = kControlBytes;
 constexpr size_t kPartialsBytes = size_t(kMaxCtas) * 3 * sizeof(double);
 constexpr size_t kExtraOffset = kPartialsOffset + kPartialsBytes;
 
+// ------------------------------------------------------------- election ----
+
+// Takes a ticket that elects the last CTA of a grid of `ctas`; returns true in the CTA that took the
+// last one.  One atomic with release and acquire semantics at GPU scope: what this CTA wrote before
+// (and, through a barrier, what its other threads wrote) is visible to whoever sees the ticket, and
+// the last CTA's later loads (again through a barrier for its other threads) see every other CTA's
+// writes -- no separate fences.  The counter wraps to 0 after the last ticket, so a workspace is
+// initialised once and reused.
+__device__ __forceinline__ bool take_last_ticket(unsigned int *ticket, unsigned int ctas) {
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(ticket), "r"(ctas - 1) : "memory");
+    return old == ctas - 1;
+}
+
 // ---------------------------------------------------------------- loads -----
 
 __device__ __forceinline__ float bf16_bits_to_float(unsigned int hi16) {

@@ -186,14 +186,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     }
     __syncthreads();
     if (tid == 0) {
-        // Ticket with release and acquire semantics at GPU scope, in place of a fence by every thread plus a
-        // relaxed atomic: the partials written above happen before it through the barrier, so they are
-        // visible to whoever sees this ticket, and the last CTA's loads below, behind the next barrier, see
-        // every other CTA's partials.  (It wraps to 0 after the last ticket: the workspace is reusable.)
-        unsigned int old;
-        asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;"
-                     : "=r"(old) : "l"(&ctl->ticket), "r"(gridDim.x - 1) : "memory");
-        is_last = (old == gridDim.x - 1);
+        is_last = take_last_ticket(&ctl->ticket, gridDim.x);
     }
     __syncthreads();
 

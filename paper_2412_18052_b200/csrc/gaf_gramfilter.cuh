@@ -449,15 +449,10 @@ __global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1)) gram_small_kern
         }
         a.partials[(size_t)threadIdx.x * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     }
-    __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int old = atomicInc(&a.replay.ctl->ticket, gridDim.x - 1);
-        is_last = (old == gridDim.x - 1);
-    }
+    if (threadIdx.x == 0) is_last = take_last_ticket(&a.replay.ctl->ticket, gridDim.x);
     __syncthreads();
     if (!is_last) return;
-    __threadfence();
 
     // last CTA: fixed-order totals (one warp per pair; all of a lane's loads are issued together,
     // this is the serial tail of the call), then the scalar walk out of shared memory

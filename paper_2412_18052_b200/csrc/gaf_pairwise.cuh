@@ -67,15 +67,10 @@ __global__ void __launch_bounds__(64 * kFinishParts) gram_finish_kernel(GramArgs
             a.gram[(size_t)j * a.K + i] = s;
         }
     }
-    __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned int old = atomicInc(&a.ctl->ticket, gridDim.x - 1);
-        is_last = (old == gridDim.x - 1);
-    }
+    if (threadIdx.x == 0) is_last = take_last_ticket(&a.ctl->ticket, gridDim.x);
     __syncthreads();
     if (!is_last) return;
-    __threadfence();
     const volatile double *G = a.gram;
     int status = 0;
     for (int idx = threadIdx.x; idx < a.K * a.K; idx += blockDim.x) {

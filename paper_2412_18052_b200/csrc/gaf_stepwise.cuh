@@ -39,13 +39,10 @@ __device__ __forceinline__ void finalize_step(const StepArgs &a, Sums3 mine, int
         a.partials[3 * blockIdx.x] = mine.p;
         a.partials[3 * blockIdx.x + 1] = mine.na;
         a.partials[3 * blockIdx.x + 2] = mine.ng;
-        __threadfence();
-        unsigned int old = atomicInc(&a.ctl->ticket, gridDim.x - 1);   // wraps to 0 after the last
-        is_last = (old == gridDim.x - 1);
+        is_last = take_last_ticket(&a.ctl->ticket, gridDim.x);
     }
     __syncthreads();
     if (!is_last || threadIdx.x >= 32) return;
-    __threadfence();
     Sums3 tot = warp_sum_partials(a.partials, gridDim.x);
     if (threadIdx.x == 0) {
         int status = 0;
@@ -187,13 +184,10 @@ __global__ void __launch_bounds__(kStepThreads, 2) cosdist_kernel(CosArgs a) {
         a.partials[3 * blockIdx.x] = blk.p;
         a.partials[3 * blockIdx.x + 1] = blk.na;
         a.partials[3 * blockIdx.x + 2] = blk.ng;
-        __threadfence();
-        unsigned int old = atomicInc(&a.ctl->ticket, gridDim.x - 1);
-        is_last = (old == gridDim.x - 1);
+        is_last = take_last_ticket(&a.ctl->ticket, gridDim.x);
     }
     __syncthreads();
     if (!is_last || threadIdx.x >= 32) return;
-    __threadfence();
     Sums3 tot = warp_sum_partials(a.partials, gridDim.x);
     if (threadIdx.x == 0) {
         int status = 0;

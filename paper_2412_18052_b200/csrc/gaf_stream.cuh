@@ -56,13 +56,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_test_kernel(StreamAr
         a.partials[3 * blockIdx.x] = blk.p;
         a.partials[3 * blockIdx.x + 1] = blk.na;
         a.partials[3 * blockIdx.x + 2] = blk.ng;
-        __threadfence();
-        const unsigned int old = atomicInc(&a.ctl->ticket, gridDim.x - 1);
-        is_last = (old == gridDim.x - 1);
+        is_last = take_last_ticket(&a.ctl->ticket, gridDim.x);
     }
     __syncthreads();
     if (!is_last || threadIdx.x >= 32) return;
-    __threadfence();
     Sums3 tot = warp_sum_partials(a.partials, gridDim.x);
     if (threadIdx.x == 0) {
         int status = 0;
