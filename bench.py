@@ -92,8 +92,8 @@ def gram_first_bytes(mask_in_order, K, D, b):
 NCU_TRAFFIC = {
     "sources": ["paper_2412_18052_b200/csrc/gaf_fused.cuh", "paper_2412_18052_b200/csrc/gaf_gramfilter.cuh",
                 "paper_2412_18052_b200/csrc/gaf_device.cuh"],
-    "sha256": "20ad1f8887539529e153445b7125b860e388b39340d38eaa53b88b2474250306",
-    "gram_fused_kernel<float,4>": {2: 233.5e6, 3: 261.6e6},
+    "sha256": "95da4a45db5cb622e2e63d7a7459a62206988c0c94e13d4d291f5692fde26e74",
+    "gram_fused_kernel<float,4>": {2: 234.2e6, 3: 261.9e6},
 }
 
 

@@ -201,9 +201,8 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
             st_relaxed_u32(&ctl->fused_word, word);
         };
         if (a.ring.K > 0) {
-            __shared__ int ring_count[kGsMaxK];
-            __shared__ unsigned long long ring_bits[kGsMaxK];
-            ring_replay_on_gram(a.ring, sgram, ring_count, ring_bits, notice);
+            __shared__ RingTable<KT> ring_table;
+            ring_replay_parallel<KT>(a.ring, sgram, ring_table, notice);
         } else {
             __shared__ ReplayTable table;
             replay_on_gram_parallel<KT>(a.replay, sgram, table, [&](unsigned long long bits) { notice(-1, bits); });

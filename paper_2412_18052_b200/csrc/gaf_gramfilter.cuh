@@ -240,6 +240,91 @@ __device__ __forceinline__ void ring_replay_on_gram(const RingArgs &r, const vol
     }
 }
 
+// The any-seed walks in table form (K <= 8), as replay_on_gram_parallel does for one order: one thread
+// per (seed, step t, accept pattern of the seed's steps 1..t-1) evaluates Eq. 4 on the Gram matrix by
+// ORIGINAL index (step v of seed s is gradient (s + v) mod K), one thread per seed then follows its
+// decisions through the table, and thread 0 picks the largest count (ties to the smallest seed) and
+// publishes.  Same sums in the same order as ring_walk_one_seed: identical outputs.
+// All threads of the block call; `early(seed, bits)` as in ring_replay_on_gram.
+template <int KT>
+struct RingTable {
+    static constexpr int kCases = (1 << (KT - 1)) - 1;          // per seed
+    float d[KT * kCases + 1];
+    unsigned char accept[KT * kCases + 1], status[KT * kCases + 1];
+    int count[KT];
+    unsigned int steps[KT];                                     // bit t-1 = step t of this seed accepted
+};
+template <int KT, typename Early = NoEarlyNotice>
+__device__ __forceinline__ void ring_replay_parallel(const RingArgs &r, const double *gram, RingTable<KT> &tb,
+                                                     Early early = Early()) {
+    constexpr int K = KT, C = RingTable<KT>::kCases;
+    for (int idx = threadIdx.x; idx < K * C; idx += blockDim.x) {
+        const int s = idx / C, cs = idx - s * C;
+        const int t = 32 - __clz(cs + 1);
+        const unsigned int m = (unsigned int)(cs + 1) - (1u << (t - 1));
+        auto in = [&](int v) { return v == 0 || ((m >> (v - 1)) & 1u); };
+        auto gi = [&](int v) { const int i = s + v; return i >= K ? i - K : i; };      // gradient of step v
+        double na = gram[s * K + s];
+#pragma unroll
+        for (int u = 1; u < K - 1; ++u) {
+            double pu = 0.0;
+#pragma unroll
+            for (int v = 0; v < u; ++v) pu += in(v) ? gram[gi(v) * K + gi(u)] : 0.0;
+            const double grown = na + 2.0 * pu + gram[gi(u) * K + gi(u)];
+            na = in(u) ? grown : na;
+        }
+        double p = 0.0;
+#pragma unroll
+        for (int v = 0; v < K - 1; ++v) p += (v < t && in(v)) ? gram[gi(v) * K + gi(t)] : 0.0;
+        int status = 0;
+        const double d = cosine_distance(p, na, gram[gi(t) * K + gi(t)], &status);
+        tb.d[idx] = (float)d;
+        tb.accept[idx] = (d <= r.tau) ? 1 : 0;
+        tb.status[idx] = (unsigned char)status;
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < K) {
+        const int s = threadIdx.x;
+        unsigned int m = 0;
+        int count = 1;
+        for (int t = 1; t < K; ++t) {
+            const int node = s * C + (1 << (t - 1)) - 1 + (int)m;
+            if (tb.accept[node]) { m |= 1u << (t - 1); ++count; }
+        }
+        tb.count[s] = count;
+        tb.steps[s] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int best = 0;
+        for (int s = 1; s < K; ++s)
+            if (tb.count[s] > tb.count[best]) best = s;
+        const unsigned int steps = tb.steps[best];
+        unsigned long long bits = 1ull << best;                 // by original index
+        for (int t = 1; t < K; ++t)
+            if ((steps >> (t - 1)) & 1u) bits |= 1ull << ((best + t) % K);
+        early(best, bits);
+        int status = 0;
+        unsigned int m = 0;
+        if (r.dist_out) r.dist_out[best] = 0.0f;
+        for (int t = 1; t < K; ++t) {
+            const int node = best * C + (1 << (t - 1)) - 1 + (int)m;
+            if (r.dist_out) r.dist_out[(best + t) % K] = tb.d[node];
+            status |= tb.status[node];
+            if (tb.accept[node]) m |= 1u << (t - 1);
+        }
+        for (int i = 0; i < K; ++i) r.mask_out[i] = (uint8_t)((bits >> i) & 1ull);
+        Control *ctl = r.ctl;
+        ctl->accept_bits = bits;
+        ctl->ring_seed = best;
+        ctl->count = tb.count[best];
+        ctl->status = status;
+        *r.count_out = tb.count[best];
+        *r.seed_out = best;
+        __threadfence();
+    }
+}
+
 // ------------------------------------------------ one-pass Gram for K <= 8 ----
 
 struct GramSmallArgs {
@@ -460,9 +545,8 @@ __global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1)) gram_small_kern
     total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
     __syncthreads();
     if (a.ring.K > 0) {
-        __shared__ int ring_count[kGsMaxK];
-        __shared__ unsigned long long ring_bits[kGsMaxK];
-        ring_replay_on_gram(a.ring, sgram, ring_count, ring_bits);
+        __shared__ RingTable<KT> ring_table;
+        ring_replay_parallel<KT>(a.ring, sgram, ring_table);
         return;
     }
     if (a.pair_dist_out == nullptr) {
