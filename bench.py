@@ -5,22 +5,32 @@
 
 One "step" is one whole gaf_filter_accumulate call over one batch of K synthetic
 micro-gradients (seed, K-1 cosine-distance tests, accepts, final division).
-The default workload is configuration 2 (ResNet18-sized gradients, D=11,227,812
+The headline workload is configuration 2 (ResNet18-sized gradients, D=11,227,812
 fp32, K=4, tau=0.97).  The path does not shard, so N > 1 runs N independent
 replicas, one per GPU (no collective on the data path); time is the max over
 ranks and the value is the aggregate over all replicas.
 
 Rank 0 prints ONE JSON line.  `value` is micro-gradient GB/s: bytes of input
 gradients consumed per second (K * elem_bytes * D per step), inputs resident in
-HBM.  `roofline` reports the HBM bytes the schedule must move (by its byte model,
-for the accept mask actually obtained) per second against the measured copy
-bandwidth of the box.  `e2e` is the same metric through the host-buffer entry
-point, pinned host memory in, results back to the host, copies inside the timed
-region.  `cpu_baseline` is the fp64 CPU oracle timed on the host cores.
+HBM.  Three byte counts are set against the measured copy bandwidth of the box,
+each under its own name in `roofline`:
+  dram_frac       bytes that really crossed HBM (ncu dram__bytes_read + dram__bytes_write of the
+                  kernels as committed, per launch) / time / peak -- the HBM utilisation;
+  min_bytes_frac  (K b + 4) D, every input read once and the output written once, / time / peak
+                  -- what any schedule must move at least;
+  model_frac      the bytes the schedule that ran asks of the memory system by its own byte model
+                  (part of which shared memory and L2 serve), / time / peak -- an effective rate.
+`roofline.frac` is dram_frac where the DRAM traffic of the kernels is on record, else
+min_bytes_frac; `roofline.basis` says which.  At N = 1 the same line carries a `configs` block with
+the other named configurations (1, 3, 4, 5), a few calls each.  `e2e` is the same metric through
+the host-buffer entry point, pinned host memory in, results back to the host, copies inside the
+timed region.  `cpu_baseline` is the fp64 CPU oracle timed on the host cores (one thread, and all
+cores).
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import statistics
@@ -33,8 +43,17 @@ sys.path.insert(0, ROOT)
 
 METRIC = "gaf_filter_accumulate micro-gradient GB/s"
 UNIT = "GB/s"
-N_SETS = 4                       # rotating input sets: each step's inputs are cold in L2
 SCHED_NAMES = {0: "auto", 1: "stepwise", 2: "gram-first, two launches", 3: "gram-first, one launch"}
+L2_BYTES = 126e6
+RAMP_SECONDS = 0.3               # back-to-back calls issued right up to every timed region
+FULL_D = {1: 1_000_000, 2: 11_227_812, 3: 11_227_812, 4: 124_439_808, 5: 1_000_000_000}
+CONFIG_K = {1: 4, 2: 4, 3: 32, 4: 8, 5: 8}
+CONFIG_B = {1: 4, 2: 4, 3: 2, 4: 4, 5: 2}
+# rotating input sets per configuration: inputs of a call were last touched n_sets - 1 calls earlier,
+# and all sets together exceed L2 (configuration 1: 12 x 16 MB), so every call starts cold in L2
+N_SETS = {1: 12, 2: 4, 4: 2, 5: 1}
+# calls timed for the entries of the `configs` block
+BLOCK_STEPS = {1: 3000, 3: 300, 4: 100, 5: 60}
 
 
 def parse_args():
@@ -44,8 +63,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5],
-                    help="named configuration (2 is the one the metric is quoted on; 3 times the "
-                         "pairwise cosine-distance matrix instead of the filter)")
+                    help="named configuration of the headline line (2 is the one the metric is quoted on; "
+                         "3 times the pairwise cosine-distance matrix instead of the filter)")
     ap.add_argument("--D", type=int, default=None,
                     help="shorter vectors of the same recipe (for profiler captures, which must stay small); "
                          "the line then says so in config.workload")
@@ -57,11 +76,15 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="leave out the `configs` block (the other named configurations)")
     return ap.parse_args()
 
 
+# ------------------------------------------------------------ byte models -----
+
 def schedule_bytes(mask_in_order, K, D, b):
-    """HBM bytes the fused streaming schedule moves for a given accept pattern:
+    """HBM bytes the fused streaming schedule asks for, for a given accept pattern:
     pass 0 reads the seed and candidate 1 and writes the running sum; pass t reads
     the running sum and candidate t+1, plus gradient t and a write-back when t was
     accepted; the last pass reads the running sum (plus the last gradient if
@@ -77,7 +100,7 @@ def schedule_bytes(mask_in_order, K, D, b):
 
 
 def gram_first_bytes(mask_in_order, K, D, b):
-    """HBM bytes of the Gram-first schedule: every gradient once for the Gram matrix,
+    """Bytes of the Gram-first schedule: every gradient once for the Gram matrix,
     the c accepted ones once more for the mean, and the output."""
     if K == 1:
         return (b + 4) * D
@@ -85,52 +108,69 @@ def gram_first_bytes(mask_in_order, K, D, b):
     return ((K + c) * b + 4) * D
 
 
-# DRAM traffic (dram__bytes_read + dram__bytes_write) of one launch of gram_fused_kernel<float,4> at
-# configuration 2, by accepted count c, from the ncu capture summarised in
-# profiles/gram_fused_config2.md.  Reported only while the kernel sources are the ones that were
-# profiled (their hash is checked); otherwise `traffic` is null.
+def min_bytes(K, D, b):
+    """What any schedule moves at least: every input once, the output once."""
+    return (K * b + 4) * D
+
+
+# DRAM traffic (ncu dram__bytes_read.sum + dram__bytes_write.sum, per launch, summed over the launches
+# of a call) of the kernels as committed, taken from the captures that the summaries in the profiler
+# folder of this repository describe.  Bytes per element index and accepted count c; a capture on a
+# shorter vector of the same recipe scales in proportion (both passes stream).  An entry is used only
+# while the listed kernel sources hash to what was profiled; otherwise `traffic` is null.
 NCU_TRAFFIC = {
-    "sources": ["paper_2412_18052_b200/csrc/gaf_fused.cuh", "paper_2412_18052_b200/csrc/gaf_gramfilter.cuh",
-                "paper_2412_18052_b200/csrc/gaf_device.cuh"],
-    "sha256": "95da4a45db5cb622e2e63d7a7459a62206988c0c94e13d4d291f5692fde26e74",
-    "gram_fused_kernel<float,4>": {2: 234.2e6, 3: 261.9e6},
+    # gram_fused_kernel<float,4> at configuration 2 itself (D = 11,227,812)
+    (2, 3): {"sources": ["gaf_fused.cuh", "gaf_gramfilter.cuh", "gaf_device.cuh"],
+             "sha256": "",
+             "bytes_per_element": {}},
 }
 
 
-def kernel_sources_hash():
+def kernel_sources_hash(names):
     import hashlib
     h = hashlib.sha256()
-    for rel in NCU_TRAFFIC["sources"]:
-        with open(os.path.join(ROOT, rel), "rb") as fh:
+    for name in names:
+        with open(os.path.join(ROOT, "paper_2412_18052_b200", "csrc", name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()
 
 
-def ncu_traffic_config2(masks, n_sets, steps):
-    """Average DRAM bytes per launch over the rotating input sets, or None."""
-    if kernel_sources_hash() != NCU_TRAFFIC["sha256"]:
+def ncu_traffic(cfg, sched_used, masks, D, n_sets, steps):
+    """Average DRAM bytes per call over the rotating input sets, or None when no capture of the
+    committed kernels is on record for this configuration and schedule."""
+    entry = NCU_TRAFFIC.get((cfg, sched_used))
+    if not entry or kernel_sources_hash(entry["sources"]) != entry["sha256"]:
         return None
-    table = NCU_TRAFFIC["gram_fused_kernel<float,4>"]
+    table = entry["bytes_per_element"]
     per_set = []
     for m in masks:
         c = sum(int(x) for x in m)
         if c not in table:
             return None
-        per_set.append(table[c])
+        per_set.append(table[c] * D)
     return sum(per_set[i % n_sets] for i in range(steps)) / steps
+
+
+def peak_bandwidth():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "of measured"
+    return 6650.0, "of fallback"
 
 
 # ---------------------------------------------------------------- clocks -----
 
-class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons of one GPU through NVML while the
-    timed region runs."""
+class Nvml:
+    """NVML handle of one GPU, initialised once, before any warm-up (initialising it with the GPU
+    idle right in front of a timed region costs the first calls of that region their clocks)."""
 
-    def __init__(self, index: int, period: float = 0.01):
-        super().__init__(daemon=True)
-        self.index, self.period = index, period
-        self.samples, self.reasons, self.max_mhz = [], set(), None
-        self._stop_evt = threading.Event()
+    REASONS = (("hw_slowdown", "nvmlClocksEventReasonHwSlowdown"),
+               ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown"),
+               ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown"),
+               ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap"),
+               ("hw_power_brake", "nvmlClocksEventReasonHwPowerBrakeSlowdown"))
+
+    def __init__(self, index: int):
         self.ok = False
         try:
             import pynvml
@@ -140,79 +180,105 @@ class ClockSampler(threading.Thread):
             self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
             self.ok = True
         except Exception:
-            self.ok = False
+            self.max_mhz = None
+
+    def read(self):
+        """(SM MHz, set of active slowdown reasons)."""
+        nv = self.nv
+        mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+        bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+        return mhz, {name for name, attr in self.REASONS if bits & getattr(nv, attr)}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons while a timed region runs."""
+
+    def __init__(self, nvml: Nvml, period: float = 0.005):
+        super().__init__(daemon=True)
+        self.nvml, self.period = nvml, period
+        self.samples, self.reasons = [], set()
+        self._stop_evt = threading.Event()
 
     def sample(self):
-        nv = self.nv
-        self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
-        bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
-        for name, bit in (("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
-                          ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
-                          ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
-                          ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap),
-                          ("hw_power_brake", nv.nvmlClocksEventReasonHwPowerBrakeSlowdown)):
-            if bits & bit:
-                self.reasons.add(name)
+        if not self.nvml.ok:
+            return
+        try:
+            mhz, reasons = self.nvml.read()
+        except Exception:
+            return
+        self.samples.append(mhz)
+        self.reasons |= reasons
 
     def run(self):
-        if not self.ok:
-            return
         while not self._stop_evt.is_set():
-            try:
-                self.sample()
-            except Exception:
-                break
+            self.sample()
             time.sleep(self.period)
 
     def stop(self):
         self._stop_evt.set()
         self.join(timeout=2)
-        if self.ok and not self.samples:
-            try:
-                self.sample()
-            except Exception:
-                pass
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "sm_max_mhz": self.nvml.max_mhz, "reasons": sorted(self.reasons),
                 "samples": len(self.samples)}
 
 
 # ---------------------------------------------------------- CPU oracle leg ---
 
-def time_oracle(cfg: int, tau: float, seconds: float):
-    """The fp64 CPU oracle, as it stands, on the same workload (single thread)."""
-    import numpy as np  # noqa: F401
-    from oracle import gaf_oracle as orc
+def oracle_sample_workload(cfg):
+    """The workload the CPU legs run: the named configuration, configurations 4 and 5 at a reduced
+    D of the same recipe so that the run stays bounded."""
     from paper_2412_18052_b200 import workloads
-
     if cfg == 3:
-        cfg = 2                     # the reference arm times the filter; 3 is the pairwise matrix
-    full = {1: 1_000_000, 2: workloads.RESNET18_100_NUMEL, 4: workloads.GPT2_SMALL_NUMEL,
-            5: 1_000_000_000}[cfg]
-    # configurations 4 and 5 are sampled at reduced D (same recipe) to bound the run
+        cfg = 2                     # the CPU legs time the filter; 3 is the pairwise matrix
+    full = FULL_D[cfg]
     D = full if cfg in (1, 2) else min(full, 32_000_000)
     w = workloads.config(cfg, device="cpu", D=None if D == full else D)
-    grads = [workloads.as_numpy_bits(g) for g in w.grads]
-    orc.filter_accumulate(grads, tau)                                  # warm (page in, compile)
-    t0 = time.perf_counter()
-    reps = 0
-    while True:
-        orc.filter_accumulate(grads, tau)
-        reps += 1
-        dt = time.perf_counter() - t0
-        if dt >= seconds or reps >= 10_000:
-            break
-    per_call = dt / reps
-    gbs = w.K * w.elem_bytes * w.D / per_call / 1e9
+    return cfg, full, w, [workloads.as_numpy_bits(g) for g in w.grads]
+
+
+def time_oracle(cfg: int, tau: float, seconds: float):
+    """The fp64 CPU oracle, as it stands, on the same workload: one thread, then the same loops split
+    over all host cores by chunks of D."""
+    from oracle import gaf_oracle as orc
+
+    cfg, full, w, grads = oracle_sample_workload(cfg)
+    gbytes = w.K * w.elem_bytes * w.D
+
+    def run(fn, budget):
+        fn()                                                       # warm (page in, compile)
+        t0 = time.perf_counter()
+        reps = 0
+        while True:
+            fn()
+            reps += 1
+            dt = time.perf_counter() - t0
+            if dt >= budget or reps >= 10_000:
+                break
+        return gbytes / (dt / reps) / 1e9, reps, dt
+
+    one, reps1, dt1 = run(lambda: orc.filter_accumulate(grads, tau), seconds)
+    cores = orc.host_cores()
+    many, repsn, dtn = run(lambda: orc.filter_accumulate_all_cores(grads, tau, n_threads=cores), seconds / 2)
     sample = (f"configuration {cfg} recipe, K={w.K}, D={w.D:,} {w.dtype}"
-              f"{'' if D == full else ' (reduced from D=%d)' % full}, whole call repeated {reps}x "
-              f"({dt:.1f} s of CPU work)")
-    return gbs, per_call, sample
+              f"{'' if w.D == full else ' (reduced from D=%d)' % full}, whole call repeated {reps1}x on one "
+              f"thread ({dt1:.1f} s) and {repsn}x on {cores} threads ({dtn:.1f} s)")
+    return {"value": one, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+            "all_cores": {"value": many, "unit": UNIT, "cores": cores,
+                          "how": "the same loops, every pass over D cut into one chunk per thread, "
+                                 "sums combined in chunk order"}}
 
 
 def workload_label(cfg, K, D, dtype, tau):
     return (f"configuration {cfg}: K={K}, D={D}, {dtype} inputs, tau={tau}, shared+private Gaussian mixture" +
             (" with ResNet18 per-tensor scales" if cfg == 2 else ""))
+
+
+def config_dict(cfg, K, D, dtype, tau, schedule, parallelism, l2, extra=None):
+    """The `config` object: the same keys from both arms."""
+    d = {"workload": workload_label(cfg, K, D, dtype, tau), "K": K, "D": D, "input_dtype": dtype, "tau": tau,
+         "schedule": schedule, "parallelism": parallelism, "l2": l2}
+    d.update(extra or {})
+    return d
 
 
 def run_reference(args):
@@ -226,11 +292,11 @@ def run_reference(args):
     from paper_2412_18052_b200 import workloads
 
     cfg = 2 if args.workload == 3 else args.workload
-    full = {1: 1_000_000, 2: workloads.RESNET18_100_NUMEL, 4: workloads.GPT2_SMALL_NUMEL, 5: 1_000_000_000}[cfg]
-    K = {1: 4, 2: 4, 4: 8, 5: 8}[cfg]
-    b = 2 if cfg == 5 else 4
+    full = FULL_D[cfg]
+    K = CONFIG_K[cfg]
+    b = CONFIG_B[cfg]
     steps, warmup = max(1, args.steps), max(0, args.warmup)
-    # about 2.2 GB/s of gradient bytes on one core: size the sample for ~100 s in all
+    # about 2 GB/s of gradient bytes on one core: size the sample for ~100 s in all
     budget_s = 100.0
     d_fit = int(budget_s / (steps + warmup) * 2.0e9 / (K * b))
     D = max(50_000, min(full, d_fit))
@@ -252,8 +318,8 @@ def run_reference(args):
         "steps": steps, "warmup": warmup, "ms_per_step": per_call * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": workload_label(cfg, K, full, w.dtype, args.tau), "K": K, "D": full,
-                   "input_dtype": w.dtype, "tau": args.tau, "sample_D": w.D},
+        "config": config_dict(cfg, K, full, w.dtype, args.tau, "CPU oracle (Algorithm 1 as written, one thread)",
+                              "host cores", f"each step runs on D={w.D} elements of the recipe"),
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -280,10 +346,204 @@ def aggregate_gbs(world: int, bytes_per_replica_step: float, ms_per_step: float)
     return world * bytes_per_replica_step / (ms_per_step * 1e-3) / 1e9
 
 
+# ------------------------------------------------------------- timing core ----
+
+def timed_region(torch, step, steps, warmup, nvml, barrier=None, ramp_seconds=RAMP_SECONDS, n_pairs=None):
+    """W warm-up calls, a ramp of back-to-back calls right up to the region, then exactly `steps`
+    calls between two events on the launching stream, bracketed by barrier + synchronize.  Clocks are
+    sampled while the region runs.  Afterwards the same calls once more with one event pair each,
+    for the median.  Returns a dict."""
+    for i in range(max(3, warmup)):
+        step(i)
+    torch.cuda.synchronize()
+    # ramp: the first calls after an idle stretch run below the steady clocks
+    ramp_calls, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < ramp_seconds:
+        for _ in range(16):
+            step(ramp_calls)
+            ramp_calls += 1
+        if ramp_calls % 256 == 0:
+            torch.cuda.synchronize()                 # bound the queue; the GPU stays busy to within one call
+    sampler = ClockSampler(nvml)
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(steps):
+        step(i)
+    ev1.record()
+    sampler.sample()                                 # the queue is still draining: a sample under load
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    clocks = sampler.stop()
+    ms_region = ev0.elapsed_time(ev1)
+    # one event pair per call (the pairs' own gaps are part of what they measure)
+    n_pairs = n_pairs or max(20, min(steps, 200))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_pairs)]
+    for i, (a, z) in enumerate(evs):
+        a.record(); step(i); z.record()
+    torch.cuda.synchronize()
+    per_call = [a.elapsed_time(z) for a, z in evs]
+    return {"ms_region": ms_region, "ms_per_step": ms_region / steps, "ramp_calls": ramp_calls,
+            "clocks": clocks, "per_call_ms": per_call}
+
+
+def fractions(ms, traffic, model_b, min_b, peak):
+    """The three byte counts over one time, as GB/s and as fractions of `peak`."""
+    def rate(nbytes):
+        return None if nbytes is None else nbytes / (ms * 1e-3) / 1e9
+    dram, model, least = rate(traffic), rate(model_b), rate(min_b)
+    return {"dram_gbs": dram, "dram_frac": None if dram is None else dram / peak,
+            "model_gbs": model, "model_frac": model / peak,
+            "min_bytes_gbs": least, "min_bytes_frac": least / peak}
+
+
+def measure_filter(torch, gaf, workloads, cfg, dev, tau, schedule, steps, warmup, nvml, rank=0, D=None,
+                   barrier=None, want_warm=False, want_c_loop=False):
+    """One named configuration of the filter on one GPU: timed region, byte counts, fractions."""
+    n_sets = N_SETS[cfg]
+    sets = [workloads.config(cfg, device=dev, seed=(cfg - 1) + 1000 * i + 17 * rank, D=D) for i in range(n_sets)]
+    w0 = sets[0]
+    K, D, b = w0.K, w0.D, w0.elem_bytes
+    dtype_code = gaf.GAF_F32 if w0.dtype == "f32" else gaf.GAF_BF16
+    ws = gaf.new_workspace(K, D, dtype_code, device=dev)
+    macro = torch.empty(D, dtype=torch.float32, device=dev)
+    mask = torch.empty(K, dtype=torch.uint8, device=dev)
+    dist_out = torch.empty(K, dtype=torch.float32, device=dev)
+    count = torch.empty(1, dtype=torch.int32, device=dev)
+
+    def step(i):
+        gaf.gaf_filter_accumulate(sets[i % n_sets].grads, tau, ws, macro_out=macro, mask_out=mask,
+                                  dist_out=dist_out, count_out=count, schedule=schedule)
+
+    # which schedule runs (the library says what its own choice was), accept pattern per input set
+    step(0)
+    sched_used = gaf.gaf_last_schedule()
+    model = gram_first_bytes if sched_used in (2, 3) else schedule_bytes
+    masks, bytes_per_set, launches_per_step = [], [], 0
+    for i in range(n_sets):
+        step(i)
+        launches_per_step = gaf.gaf_last_launch_count()
+        torch.cuda.synchronize()
+        m = mask.cpu().tolist()
+        masks.append(m)
+        bytes_per_set.append(model(m, K, D, b))
+    status = gaf.gaf_read_status(ws)
+
+    t = timed_region(torch, step, steps, warmup, nvml, barrier)
+    grad_bytes = K * b * D
+    model_b = sum(bytes_per_set[i % n_sets] for i in range(steps)) / steps
+    out = {"K": K, "D": D, "b": b, "dtype": w0.dtype, "n_sets": n_sets, "grad_bytes": grad_bytes, "masks": masks,
+           "sched_used": sched_used, "launches_per_step": launches_per_step, "status": status,
+           "model_bytes": model_b, "min_bytes": min_bytes(K, D, b),
+           "traffic": ncu_traffic(cfg, sched_used, masks, D, n_sets, steps) if abs(tau - 0.97) < 1e-12 else None,
+           "timing": t, "sets": sets, "ws": ws, "outputs": (macro, mask, dist_out, count), "dtype_code": dtype_code}
+
+    if want_warm:
+        # the same input set every call: whatever of it fits stays in L2 between calls
+        n_warm = min(max(steps, 200), 500)
+        for _ in range(5):
+            step(0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n_warm):
+            step(0)
+        e1.record()
+        torch.cuda.synchronize()
+        warm_ms = e0.elapsed_time(e1) / n_warm
+        out["warm_l2"] = {"ms_per_step": warm_ms, "value": grad_bytes / (warm_ms * 1e-3) / 1e9, "unit": UNIT,
+                          "steps": n_warm,
+                          "note": "one input set repeated: whatever of it fits stays in L2 between calls; "
+                                  "not the headline"}
+    if want_c_loop:
+        # the same calls issued by a loop in C inside the library: the interpreter's per-call cost is out
+        n_c = max(steps, 1000)
+        grads_sets = [s.grads for s in sets]
+        gaf.gaf_filter_accumulate_repeat(200, grads_sets, tau, ws, macro, mask, dist_out, count, schedule=schedule)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        gaf.gaf_filter_accumulate_repeat(n_c, grads_sets, tau, ws, macro, mask, dist_out, count, schedule=schedule)
+        e1.record()
+        torch.cuda.synchronize()
+        out["c_loop"] = {"ms_per_step": e0.elapsed_time(e1) / n_c, "steps": n_c,
+                         "note": "the same calls from a loop in C (gaf_filter_accumulate_repeat)"}
+    return out
+
+
+def block_entry(m, peak, peak_kind, tau, schedule):
+    """One entry of the `configs` block from a measure_filter result."""
+    t = m["timing"]
+    ms = t["ms_per_step"]
+    fr = fractions(ms, m["traffic"], m["model_bytes"], m["min_bytes"], peak)
+    per_call = t["per_call_ms"]
+    mhz = t["clocks"]["sm_mhz"]
+    e = {"workload": workload_label(m["cfg"], m["K"], m["D"], m["dtype"], tau),
+         "schedule": SCHED_NAMES[schedule] + (" -> " + SCHED_NAMES[m["sched_used"]] if not schedule else ""),
+         "steps": m["steps"], "ramp_calls": t["ramp_calls"], "ms_per_call": ms,
+         "ms_per_call_median_of_event_pairs": statistics.median(per_call), "event_pairs": len(per_call),
+         "value": m["grad_bytes"] / (ms * 1e-3) / 1e9, "unit": UNIT,
+         "launches_per_call": m["launches_per_step"], "accept_masks": m["masks"],
+         "l2": f"{m['n_sets']} rotating input sets of {m['grad_bytes'] / 1e6:.0f} MB each"
+               if m["n_sets"] > 1 else f"inputs of one call ({m['grad_bytes'] / 1e9:.1f} GB) exceed L2",
+         "model_bytes_per_call": m["model_bytes"], "min_bytes_per_call": m["min_bytes"],
+         "traffic": m["traffic"], "peak": peak, "peak_kind": peak_kind, "clocks": t["clocks"],
+         "ms_x_sm_mhz": None if mhz is None else ms * mhz}
+    e.update(fr)
+    for key in ("warm_l2", "c_loop"):
+        if key in m:
+            e[key] = m[key]
+    return e
+
+
+def measure_pairwise(torch, gaf, workloads, dev, steps, warmup, nvml, K=None, D=None, fp32=False):
+    """Configuration 3: the K x K pairwise cosine-distance matrix."""
+    w = workloads.config(3, device=dev, K=K, D=D)
+    if fp32:
+        w = workloads.mixture(w.K, w.D, "f32", w.rho, w.seed, device=dev)
+    K, D, b = w.K, w.D, w.elem_bytes
+    ws = gaf.new_workspace(K, D, gaf.GAF_F32 if fp32 else gaf.GAF_BF16, device=dev)
+    dist_out = torch.empty(K, K, dtype=torch.float32, device=dev)
+    gram = torch.empty(K, K, dtype=torch.float64, device=dev)
+
+    def step(_i):
+        gaf.gaf_pairwise_cosdist(w.grads, ws, dist_out=dist_out, gram_out=gram)
+
+    step(0)
+    launches = gaf.gaf_last_launch_count()
+    t = timed_region(torch, step, steps, warmup, nvml)
+    return {"K": K, "D": D, "b": b, "dtype": w.dtype, "grad_bytes": K * b * D, "launches": launches, "timing": t,
+            "kernel": ("gram_tc_kernel" if (not fp32 and 8 < K <= 64) else
+                       "gram_panel_kernel" if K > 8 else "gram_small_kernel") + " + finishing (whole call)"}
+
+
+def pairwise_entry(m, peak, peak_kind, steps):
+    t = m["timing"]
+    ms = t["ms_per_step"]
+    achieved = m["grad_bytes"] / (ms * 1e-3) / 1e9
+    mhz = t["clocks"]["sm_mhz"]
+    return {"workload": f"configuration 3: pairwise matrix, K={m['K']}, D={m['D']}, {m['dtype']} inputs",
+            "op": "gaf_pairwise_cosdist", "steps": steps, "ramp_calls": t["ramp_calls"], "ms_per_call": ms,
+            "ms_per_call_median_of_event_pairs": statistics.median(t["per_call_ms"]),
+            "event_pairs": len(t["per_call_ms"]), "value": achieved, "unit": UNIT,
+            "launches_per_call": m["launches"], "kernel": m["kernel"],
+            "l2": f"inputs of one call ({m['grad_bytes'] / 1e6:.0f} MB) exceed the 126 MB L2",
+            "model_bytes_per_call": m["grad_bytes"], "min_bytes_per_call": m["grad_bytes"],
+            "byte_model": "every gradient read once: K b D (= the minimum)",
+            "model_gbs": achieved, "model_frac": achieved / peak, "min_bytes_gbs": achieved,
+            "min_bytes_frac": achieved / peak, "dram_gbs": None, "dram_frac": None, "traffic": None,
+            "peak": peak, "peak_kind": peak_kind, "clocks": t["clocks"],
+            "ms_x_sm_mhz": None if mhz is None else ms * mhz}
+
+
 # ------------------------------------------------------------------ ours -----
 
 def run_pairwise(args):
-    """Configuration 3: the K x K pairwise cosine-distance matrix (one GPU)."""
+    """--workload 3: the pairwise matrix as the headline line (one GPU)."""
     import torch
 
     import paper_2412_18052_b200 as gaf
@@ -292,55 +552,27 @@ def run_pairwise(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(0)
-    w = workloads.config(3, device="cuda:0", K=args.K, D=args.D)
+    nvml = Nvml(0)
     named = args.K is None and args.D is None and not args.fp32
-    if args.fp32:
-        w = workloads.mixture(w.K, w.D, "f32", w.rho, w.seed, device="cuda:0")
-    K, D, b = w.K, w.D, w.elem_bytes
-    ws = gaf.new_workspace(K, D, gaf.GAF_F32 if args.fp32 else gaf.GAF_BF16, device="cuda:0")
-    dist_out = torch.empty(K, K, dtype=torch.float32, device="cuda:0")
-    gram = torch.empty(K, K, dtype=torch.float64, device="cuda:0")
-
-    def step():
-        gaf.gaf_pairwise_cosdist(w.grads, ws, dist_out=dist_out, gram_out=gram)
-
-    for _ in range(max(3, args.warmup)):
-        step()
-    launches = gaf.gaf_last_launch_count()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(0)
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1) / args.steps
-    in_bytes = K * b * D
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_kind = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-    else:
-        peak, peak_kind = 6650.0, "fallback"
-    achieved = in_bytes / (ms * 1e-3) / 1e9
+    m = measure_pairwise(torch, gaf, workloads, "cuda:0", args.steps, args.warmup, nvml, K=args.K, D=args.D,
+                         fp32=args.fp32)
+    peak, peak_kind = peak_bandwidth()
+    e = pairwise_entry(m, peak, peak_kind, args.steps)
+    K = m["K"]
     line = {
-        "metric": "gaf_pairwise_cosdist micro-gradient GB/s", "value": achieved, "unit": UNIT, "n_gpus": 1,
-        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32 products, f64 sums" if (args.fp32 or K > 32) else "bf16 x bf16 -> f32 (tensor cores), f64 sums",
+        "metric": "gaf_pairwise_cosdist micro-gradient GB/s", "value": e["value"], "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": e["ms_per_call"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 products, f64 sums" if (args.fp32 or K > 64) else "bf16 x bf16 -> f32 (tensor cores), f64 sums",
         "data": "synthetic",
-        "config": {"workload": f"configuration 3: pairwise matrix, K={K}, D={D}, {w.dtype} inputs" +
-                               ("" if named else " (NOT the named configuration: size or type overridden)"),
-                   "K": K, "D": D,
-                   "l2": f"inputs of one call ({in_bytes / 1e6:.0f} MB) exceed the 126 MB L2"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": f"of {peak_kind}",
-                     "kernel": ("gram_tc_kernel" if (not args.fp32 and 8 < K <= 32) else
-                                "gram_panel_kernel" if K > 8 else "gram_small_kernel") + " + finishing (whole call)",
-                     "byte_model": "every gradient read once: K b D", "algorithmic_bytes_per_launch": in_bytes},
-        "e2e": None, "gpu_launches": launches * args.steps, "clocks": clocks, "cpu_baseline": None,
+        "config": {"workload": e["workload"] + ("" if named else " (NOT the named configuration: size or type overridden)"),
+                   "K": K, "D": m["D"], "l2": e["l2"]},
+        "roofline": {"bound": "hbm", "achieved": e["value"], "peak": peak, "unit": "GB/s", "frac": e["value"] / peak,
+                     "basis": "min_bytes (= byte model: every gradient read once)", "traffic": None,
+                     "peak_kind": peak_kind, "kernel": m["kernel"], "algorithmic_bytes_per_launch": m["grad_bytes"],
+                     "model_frac": e["model_frac"], "min_bytes_frac": e["min_bytes_frac"], "dram_frac": None},
+        "ramp_calls": e["ramp_calls"], "ms_per_call_median_of_event_pairs": e["ms_per_call_median_of_event_pairs"],
+        "e2e": None, "gpu_launches": m["launches"] * args.steps, "clocks": e["clocks"], "cpu_baseline": None,
     }
     print(json.dumps(line), flush=True)
 
@@ -359,121 +591,40 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
+    nvml = Nvml(local)                        # before any warm-up
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
-
-    cfg = args.workload
-    n_sets = N_SETS if cfg in (1, 2) else (2 if cfg == 4 else 1)
-    sets = [workloads.config(cfg, device=dev, seed=(cfg - 1) + 1000 * i + 17 * rank, D=args.D)
-            for i in range(n_sets)]
-    w0 = sets[0]
-    K, D, b = w0.K, w0.D, w0.elem_bytes
-    dtype_code = gaf.GAF_F32 if w0.dtype == "f32" else gaf.GAF_BF16
-    ws = gaf.new_workspace(K, D, dtype_code, device=dev)
-    macro = torch.empty(D, dtype=torch.float32, device=dev)
-    mask = torch.empty(K, dtype=torch.uint8, device=dev)
-    dist_out = torch.empty(K, dtype=torch.float32, device=dev)
-    count = torch.empty(1, dtype=torch.int32, device=dev)
-
-    def step(i):
-        gaf.gaf_filter_accumulate(sets[i % n_sets].grads, args.tau, ws, macro_out=macro, mask_out=mask,
-                                  dist_out=dist_out, count_out=count, schedule=args.schedule)
-
-    # which schedule runs (the library says what its own choice was) and its byte model
-    step(0)
-    sched_used = gaf.gaf_last_schedule()
-    model = gram_first_bytes if sched_used in (2, 3) else schedule_bytes
-    # accept pattern and byte model per input set (also a warm-up)
-    masks, bytes_per_set, launches_per_step = [], [], 0
-    for i in range(n_sets):
-        step(i)
-        launches_per_step = gaf.gaf_last_launch_count()
-        torch.cuda.synchronize()
-        m = mask.cpu().tolist()
-        masks.append(m)
-        bytes_per_set.append(model(m, K, D, b))
-    for i in range(max(3, args.warmup)):
-        step(i)
-    torch.cuda.synchronize()
 
     def barrier():
         if world > 1:
             dist.barrier()
 
-    steps = args.steps
-    sampler = ClockSampler(local)
-    barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for i in range(steps):
-        step(i)
-    ev1.record()
-    torch.cuda.synchronize()
-    barrier()
-    clocks = sampler.stop()
-    elapsed_ms = max_over_ranks(ev0.elapsed_time(ev1), dev)
-    ms_per_step = elapsed_ms / steps
-    grad_bytes = K * b * D
+    cfg, steps = args.workload, args.steps
+    peak, peak_kind = peak_bandwidth()
+    m = measure_filter(torch, gaf, workloads, cfg, dev, args.tau, args.schedule, steps, args.warmup, nvml,
+                       rank=rank, D=args.D, barrier=barrier, want_warm=cfg in (1, 2))
+    t = m["timing"]
+    K, D, b, grad_bytes = m["K"], m["D"], m["b"], m["grad_bytes"]
+    ms_per_step = max_over_ranks(t["ms_region"], dev) / steps
     value = aggregate_gbs(world, grad_bytes, ms_per_step)
-
-    # dominant kernel, timed per launch with events on the launching stream
-    n_launch_timed = min(steps, 200)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-           for _ in range(n_launch_timed)]
-    for i, (a, z) in enumerate(evs):
-        a.record(); step(i); z.record()
-    torch.cuda.synchronize()
-    launch_ms = [a.elapsed_time(z) for a, z in evs]
-    avg_launch_ms = sum(launch_ms) / len(launch_ms)
-    avg_bytes = sum(bytes_per_set[i % n_sets] for i in range(n_launch_timed)) / n_launch_timed
-
-    # "warm" figure for the configurations that partly live in L2: the same input set every call
-    warm = None
-    if n_sets > 1 and cfg in (1, 2):
-        n_warm = min(steps, 500)
-        for _ in range(5):
-            step(0)
-        wev0, wev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        wev0.record()
-        for _ in range(n_warm):
-            step(0)
-        wev1.record()
-        torch.cuda.synchronize()
-        warm_ms = wev0.elapsed_time(wev1) / n_warm
-        warm = {"ms_per_step": warm_ms, "value": grad_bytes / (warm_ms * 1e-3) / 1e9, "unit": UNIT, "steps": n_warm,
-                "note": "one input set repeated: whatever of it fits stays in L2 between calls; not the headline"}
-
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_kind = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-    else:
-        peak, peak_kind = 6650.0, "fallback"
-    # Roofline figure: algorithmic bytes per call over the average duration of a call inside the timed
-    # region (events on the launching stream around the K back-to-back calls).  With the one-launch
-    # schedule a call IS one kernel launch.  The same ratio from one event pair per call is kept beside
-    # it: it also contains the event records' own gaps.
-    region_bytes = sum(bytes_per_set[i % n_sets] for i in range(steps)) / steps
-    achieved = region_bytes / (ms_per_step * 1e-3) / 1e9
-    per_call_events = avg_bytes / (avg_launch_ms * 1e-3) / 1e9
+    fr = fractions(ms_per_step, m["traffic"], m["model_bytes"], m["min_bytes"], peak)
+    per_call = t["per_call_ms"]
 
     # end to end through the host-buffer entry point
     e2e = None
     if args.e2e_steps > 0:
         n_e2e = args.e2e_steps
-        host_sets = [[g.cpu().pin_memory() for g in s.grads] for s in sets[:2]]
-        staging = torch.empty(gaf.gaf_host_staging_bytes(K, D, dtype_code), dtype=torch.uint8, device=dev)
+        host_sets = [[g.cpu().pin_memory() for g in s.grads] for s in m["sets"][:2]]
+        staging = torch.empty(gaf.gaf_host_staging_bytes(K, D, m["dtype_code"]), dtype=torch.uint8, device=dev)
         macro_h = torch.empty(D, dtype=torch.float32).pin_memory()
         mask_h = torch.empty(K, dtype=torch.uint8).pin_memory()
         dist_h = torch.empty(K, dtype=torch.float32).pin_memory()
         count_h = torch.empty(1, dtype=torch.int32).pin_memory()
 
         def e2e_step(i):
-            gaf.gaf_filter_accumulate_host(host_sets[i % len(host_sets)], args.tau, staging, ws, macro_h,
+            gaf.gaf_filter_accumulate_host(host_sets[i % len(host_sets)], args.tau, staging, m["ws"], macro_h,
                                            mask_h, dist_h, count_h, schedule=args.schedule)
-        for i in range(2):
+        for i in range(3):
             e2e_step(i)
         barrier()
         torch.cuda.synchronize()
@@ -485,50 +636,88 @@ def run_ours(args):
         e2e = {"value": aggregate_gbs(world, grad_bytes, dt / n_e2e * 1e3), "unit": UNIT,
                "h2d_bytes_per_step": grad_bytes, "d2h_bytes_per_step": 4 * D + K + 4 * K + 4,
                "steps": n_e2e}
+        del host_sets, staging, macro_h, e2e_step
+
+    # the other named configurations, a few calls each (one GPU, the default line only)
+    block = None
+    if world == 1 and cfg == 2 and args.D is None and not args.no_configs:
+        sched_used_main = m["sched_used"]
+        m_keep = {k: v for k, v in m.items() if k not in ("sets", "ws", "outputs")}
+        del m
+        gc.collect()
+        torch.cuda.empty_cache()
+        m = m_keep
+        m["sched_used"] = sched_used_main
+        block = {}
+        for c in (1, 3, 4, 5):
+            try:
+                if c == 3:
+                    r = measure_pairwise(torch, gaf, workloads, dev, BLOCK_STEPS[3], 5, nvml)
+                    block["3"] = pairwise_entry(r, peak, peak_kind, BLOCK_STEPS[3])
+                else:
+                    r = measure_filter(torch, gaf, workloads, c, dev, 0.97, 0, BLOCK_STEPS[c], 5, nvml,
+                                       want_warm=(c == 1), want_c_loop=(c == 1))
+                    r["cfg"], r["steps"] = c, BLOCK_STEPS[c]
+                    block[str(c)] = block_entry(r, peak, peak_kind, 0.97, 0)
+            except Exception as exc:      # a configuration that cannot run here is reported, not hidden
+                block[str(c)] = {"error": f"{type(exc).__name__}: {exc}"}
+            r = None
+            gc.collect()
+            torch.cuda.empty_cache()
 
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            gbs, per_call, sample = time_oracle(cfg, args.tau, args.cpu_seconds)
-            cpu = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}
+            cpu = time_oracle(cfg, args.tau, args.cpu_seconds)
+        sched_used = m["sched_used"]
+        n_sets = m["n_sets"]
+        basis = "dram" if fr["dram_frac"] is not None else "min_bytes"
+        achieved = fr["dram_gbs"] if basis == "dram" else fr["min_bytes_gbs"]
+        mhz = t["clocks"]["sm_mhz"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {
-                "workload": workload_label(cfg, K, D, w0.dtype, args.tau) +
-                            (" (REDUCED length, not the named configuration)" if args.D else ""),
-                "K": K, "D": D, "input_dtype": w0.dtype, "tau": args.tau,
-                "schedule": SCHED_NAMES[args.schedule] +
-                            (" -> " + SCHED_NAMES[sched_used] if not args.schedule else ""),
-                "parallelism": "replicas only (the path does not shard)" if world > 1 else "1 GPU",
-                "l2": f"{n_sets} rotating input sets of {grad_bytes / 1e6:.0f} MB each (inputs of a step "
-                      f"exceed the 126 MB L2 and were last touched {n_sets - 1} steps earlier)"
-                      if n_sets > 1 else f"inputs of one step ({grad_bytes / 1e9:.1f} GB) exceed L2",
-                "accept_masks": masks,
-            },
+            "config": config_dict(
+                cfg, K, D, m["dtype"], args.tau,
+                SCHED_NAMES[args.schedule] + (" -> " + SCHED_NAMES[sched_used] if not args.schedule else ""),
+                "replicas only (the path does not shard)" if world > 1 else "1 GPU",
+                (f"{n_sets} rotating input sets of {grad_bytes / 1e6:.0f} MB each (inputs of a step "
+                 f"exceed the 126 MB L2 and were last touched {n_sets - 1} steps earlier)"
+                 if n_sets > 1 and grad_bytes > L2_BYTES else
+                 f"{n_sets} rotating input sets of {grad_bytes / 1e6:.0f} MB each ({n_sets * grad_bytes / 1e6:.0f} MB "
+                 f"in all, more than the 126 MB L2)" if n_sets > 1 else
+                 f"inputs of one step ({grad_bytes / 1e9:.1f} GB) exceed L2"),
+                {"accept_masks": m["masks"],
+                 **({"note": "REDUCED length, not the named configuration"} if args.D else {})}),
             "roofline": {
-                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0,
-                "traffic": (ncu_traffic_config2(masks, n_sets, steps)
-                            if (cfg == 2 and sched_used == 3 and abs(args.tau - 0.97) < 1e-12) else None),
-                "peak_kind": f"of {peak_kind}",
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "basis": ("dram: bytes that crossed HBM per call (ncu, `traffic`) / time" if basis == "dram" else
+                          "min_bytes: (K b + 4) D / time (no DRAM traffic on record for the kernels as committed)"),
+                "traffic": m["traffic"], "peak_kind": peak_kind,
+                "dram_frac": fr["dram_frac"], "min_bytes_frac": fr["min_bytes_frac"], "model_frac": fr["model_frac"],
+                "dram_gbs": fr["dram_gbs"], "min_bytes_gbs": fr["min_bytes_gbs"], "model_gbs": fr["model_gbs"],
+                "frac_of_nominal_8000": achieved / 8000.0,
                 "kernel": {3: "gram_fused_kernel (the whole call is this one launch)",
                            2: "Gram kernel + masked_mean_kernel (whole call, both HBM-streaming)",
-                           1: "step_kernel x%d (whole call)" % launches_per_step}[sched_used],
-                "byte_model": ("Gram-first: ((K + c) b + 4) D" if sched_used in (2, 3)
+                           1: "step_kernel x%d (whole call)" % m["launches_per_step"]}[sched_used],
+                "byte_model": ("Gram-first: ((K + c) b + 4) D; part of it is served by shared memory and L2, "
+                               "so model_frac is an effective rate, not HBM utilisation" if sched_used in (2, 3)
                                else "streaming: (2b+4) + sum_t [4 + b + a_t (b+4)] + 8 + a_last b, times D"),
-                "algorithmic_bytes_per_launch": region_bytes, "avg_launch_ms": ms_per_step,
-                "launches_per_call": launches_per_step,
-                "per_call_event_pairs": {"achieved": per_call_events, "frac": per_call_events / peak,
-                                         "avg_call_ms": avg_launch_ms, "calls": n_launch_timed},
-                "min_bytes_per_step": (K * b + 4) * D,
+                "model_bytes_per_launch": m["model_bytes"], "min_bytes_per_step": m["min_bytes"],
+                "algorithmic_bytes_per_launch": m["min_bytes"],
+                "avg_launch_ms": ms_per_step, "launches_per_call": m["launches_per_step"],
+                "per_call_event_pairs": {"median_ms": statistics.median(per_call),
+                                         "mean_ms": sum(per_call) / len(per_call), "calls": len(per_call)},
+                "ms_x_sm_mhz": None if mhz is None else ms_per_step * mhz,
             },
+            "ramp_calls": t["ramp_calls"],
             "e2e": e2e,
-            "warm_l2": warm,
-            "gpu_launches": launches_per_step * steps,
-            "clocks": clocks,
+            "warm_l2": m.get("warm_l2"),
+            "gpu_launches": m["launches_per_step"] * steps,
+            "clocks": t["clocks"],
             "cpu_baseline": cpu,
+            "configs": block,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

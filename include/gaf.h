@@ -97,9 +97,17 @@ enum {
 enum {
     GAF_STATUS_ZERO_NORM = 1,   /* some tested pair had a zero norm (distance set to 1) */
     GAF_STATUS_NONFINITE = 2,   /* some sum was NaN or Inf */
-    GAF_STATUS_TIMEOUT = 4      /* a bounded wait inside a kernel (tensor-core Gram pipeline,
+    GAF_STATUS_TIMEOUT = 4,     /* a bounded wait inside a kernel (tensor-core Gram pipeline,
                                    one-launch Gram-first schedule) ran out; the outputs of that
                                    call are not valid */
+    GAF_STATUS_ILL_CONDITIONED = 8  /* after some accept the running sum g of the c accepted gradients
+                                   had c * sum_i |g_i|^2 > 167 |g|^2: the accepted gradients nearly
+                                   cancel (only possible with tau > 1, when a gradient that points
+                                   against the sum is accepted).  |g|^2 is then a small difference of
+                                   large binary32-rounded terms and neither the 1e-5 on the distances
+                                   of Eq. 4 nor the 1e-6 on the binary32 macro-gradient is guaranteed
+                                   from that step on.  The outputs are still what the arithmetic
+                                   gave; not an error. */
 };
 
 /* Human-readable name of a return code.  Host only; never NULL. */
@@ -164,6 +172,23 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
                           int32_t *count_out,
                           void *workspace, size_t workspace_bytes,
                           int schedule, void *cuda_stream);
+
+/*
+ * The same call `repeats` times back to back on the stream, cycling through `n_sets` sets of
+ * inputs (call r reads set r mod n_sets): exactly what a host loop in C around
+ * gaf_filter_accumulate does, for callers -- benchmarks above all -- driven from an interpreted
+ * language whose own per-call cost would otherwise be measured instead of the library's.  Every
+ * repetition overwrites the same outputs; gaf_last_launch_count() reports the launches of all
+ * repetitions together.
+ *   grads       HOST array of n_sets * K device pointers, set after set
+ *   repeats     >= 0;  n_sets >= 1;  everything else as in gaf_filter_accumulate
+ */
+int gaf_filter_accumulate_repeat(int repeats, int n_sets, const void *const *grads, int K, int64_t D,
+                                 int dtype, double tau, const int32_t *order,
+                                 float *macro_out, uint8_t *mask_out, float *dist_out,
+                                 int32_t *count_out,
+                                 void *workspace, size_t workspace_bytes,
+                                 int schedule, void *cuda_stream);
 
 /*
  * Order-indifferent variant, as sketched at the end of Section 3.1: Algorithm 1 is
@@ -308,12 +333,30 @@ int gaf_cosdist_static(const void *x, const void *y, int64_t D, int dtype,
                        float *dist_out, double *stats_out, void *cuda_stream);
 
 /* Number of kernel launches the most recent gaf_* call of this thread issued
- * (host-side counter, for benchmarks). */
+ * (host-side counter, for benchmarks; gaf_cosdist_static counts too). */
 int gaf_last_launch_count(void);
 
 /* The GAF_SCHED_* value the most recent gaf_filter_accumulate call of this thread ran with
  * (what GAF_SCHED_AUTO resolved to).  Host-side, for benchmarks and tests. */
 int gaf_last_schedule(void);
+
+/*
+ * Test hook for the bounded waits inside the kernels (failure detection without a faulted GPU).
+ * Two kernels wait on something another part of the same launch produces: the one-launch
+ * Gram-first schedule (its CTAs poll one word for the decisions) and the tensor-core Gram
+ * pipeline (mbarrier waits between loaders, MMA issuer and epilogue).  Every such wait gives up
+ * after a fixed number of attempts -- seconds in normal use, never reached -- raises
+ * GAF_STATUS_TIMEOUT and lets the kernel return in an orderly way (copies in flight are awaited,
+ * tensor memory is freed).  This call lets a test see that path run, for the following launches of
+ * the calling thread:
+ *   wait_limit   attempts before a wait gives up; 0 restores the built-in limits
+ *   withhold     non-zero: the awaited signal is never given (the deciding CTA does not publish the
+ *                decision word; the first tile's barrier expects one arrival more than will come),
+ *                so that every wait runs out.  Nothing traps and nothing waits without a limit.
+ * The outputs of a call made with `withhold` set are not valid; the workspace stays usable: the next
+ * ordinary call on it is correct.  Always returns GAF_OK.  Off by default; not for production use.
+ */
+int gaf_test_set_wait_fault(unsigned int wait_limit, int withhold);
 
 #ifdef __cplusplus
 }

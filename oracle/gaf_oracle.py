@@ -26,7 +26,10 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "gaf_oracle.c")
 _LIB = os.path.join(_HERE, "libgaf_oracle.so")
+_SRC_MT = os.path.join(_HERE, "gaf_oracle_mt.c")
+_LIB_MT = os.path.join(_HERE, "libgaf_oracle_mt.so")
 _lib = None
+_lib_mt = None
 _lib_override = None   # set by tests that load a deliberately broken copy
 
 
@@ -34,8 +37,8 @@ def compile_c(src: str, lib: str) -> str:
     """gcc, no fast-math: every sum keeps the order it is written in."""
     tmp = lib + f".{os.getpid()}.tmp"
     subprocess.check_call(
-        ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fno-fast-math",
-         "-o", tmp, src, "-lm"])
+        ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fno-fast-math", "-pthread",
+         "-I", _HERE, "-o", tmp, src, "-lm"])
     os.replace(tmp, lib)
     return lib
 
@@ -45,6 +48,10 @@ def build(force: bool = False) -> str:
     stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
     if force or stale:
         compile_c(_SRC, _LIB)
+    # the several-threads form of the filter (gaf_oracle_mt.c includes gaf_oracle.c)
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_MT))
+    if force or (not os.path.exists(_LIB_MT)) or os.path.getmtime(_LIB_MT) < newest:
+        compile_c(_SRC_MT, _LIB_MT)
     return _LIB
 
 
@@ -154,6 +161,46 @@ def filter_accumulate(grads: Sequence[np.ndarray], tau: float,
     if rc != 0:
         raise ValueError("oracle rejected its arguments")
     return FilterResult(out, mask, dist, int(count.value), stats)
+
+
+def filter_accumulate_all_cores(grads: Sequence[np.ndarray], tau: float,
+                                order: Optional[Sequence[int]] = None,
+                                n_threads: Optional[int] = None) -> FilterResult:
+    """The same Algorithm 1 + Eq. 5 with every pass over the D parameters split into
+    ``n_threads`` consecutive chunks (default: the cores this process may run on), the sums
+    of each test combined in chunk order.  For the all-cores CPU baseline of the benchmark."""
+    global _lib_mt
+    if _lib_mt is None:
+        build()
+        lib = ctypes.CDLL(_LIB_MT)
+        vp, i64, i32, dbl = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_double
+        lib.gaf_oracle_filter_accumulate_mt.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, i32]
+        lib.gaf_oracle_filter_accumulate_mt.restype = ctypes.c_int
+        _lib_mt = lib
+    if n_threads is None:
+        n_threads = host_cores()
+    arrs, ptrs, code, D = _prep(grads)
+    K = len(arrs)
+    order_arr = None if order is None else np.ascontiguousarray(order, dtype=np.int32)
+    out = np.empty(D, dtype=np.float64)
+    mask = np.zeros(K, dtype=np.uint8)
+    dist = np.zeros(K, dtype=np.float64)
+    count = ctypes.c_int32()
+    rc = _lib_mt.gaf_oracle_filter_accumulate_mt(
+        ctypes.cast(ptrs, ctypes.c_void_p), K, D, code, float(tau),
+        None if order_arr is None else order_arr.ctypes.data,
+        out.ctypes.data, mask.ctypes.data, dist.ctypes.data, ctypes.addressof(count), int(n_threads))
+    if rc != 0:
+        raise ValueError("oracle rejected its arguments or could not start its threads")
+    return FilterResult(out, mask, dist, int(count.value), np.zeros((K, 3)))
+
+
+def host_cores() -> int:
+    """Cores this process may run on."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return max(1, os.cpu_count() or 1)
 
 
 def filter_any_seed(grads: Sequence[np.ndarray], tau: float):

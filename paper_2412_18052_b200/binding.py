@@ -14,7 +14,7 @@ import torch
 
 GAF_F32, GAF_BF16 = 0, 1
 GAF_SCHED_AUTO, GAF_SCHED_STEPWISE, GAF_SCHED_GRAM, GAF_SCHED_GRAM_FUSED = 0, 1, 2, 3
-GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT = 1, 2, 4
+GAF_STATUS_ZERO_NORM, GAF_STATUS_NONFINITE, GAF_STATUS_TIMEOUT, GAF_STATUS_ILL_CONDITIONED = 1, 2, 4, 8
 GAF_MAX_K = 64
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgaf.so")
@@ -25,7 +25,8 @@ EXPORTS = [
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
     "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
     "gaf_filter_accumulate_any_seed", "gaf_stream_begin", "gaf_stream_push", "gaf_stream_end",
-    "gaf_filter_accumulate_bucketed", "gaf_last_schedule",
+    "gaf_filter_accumulate_bucketed", "gaf_last_schedule", "gaf_test_set_wait_fault",
+    "gaf_filter_accumulate_repeat",
 ]
 
 
@@ -52,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.gaf_workspace_init.argtypes = [vp, sz, vp]
         L.gaf_cosdist.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
         L.gaf_filter_accumulate.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, i32, vp]
+        L.gaf_filter_accumulate_repeat.argtypes = [i32, i32, vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz,
+                                                   i32, vp]
         L.gaf_host_staging_bytes.argtypes = [i32, i64, i32, ctypes.POINTER(sz)]
         L.gaf_filter_accumulate_host.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz,
                                                  vp, sz, i32, vp]
@@ -59,6 +62,7 @@ def lib() -> ctypes.CDLL:
         L.gaf_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.gaf_last_launch_count.argtypes = []
         L.gaf_last_schedule.argtypes = []
+        L.gaf_test_set_wait_fault.argtypes = [ctypes.c_uint, i32]
         L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.gaf_filter_accumulate_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, vp]
         L.gaf_filter_accumulate_bucketed.argtypes = [vp, i32, i64, i32, dbl, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -183,6 +187,23 @@ def gaf_filter_accumulate(grads: Sequence[torch.Tensor], tau: float, workspace: 
     return macro_out, mask_out, dist_out, count_out
 
 
+def gaf_filter_accumulate_repeat(repeats: int, sets: Sequence[Sequence[torch.Tensor]], tau: float,
+                                 workspace: torch.Tensor, macro_out: torch.Tensor, mask_out: torch.Tensor,
+                                 dist_out: torch.Tensor, count_out: torch.Tensor,
+                                 order: Optional[Sequence[int]] = None, schedule: int = GAF_SCHED_AUTO) -> None:
+    """``repeats`` calls of gaf_filter_accumulate issued by one C loop, call r on ``sets[r % len(sets)]``."""
+    K, D = len(sets[0]), sets[0][0].numel()
+    flat = [g for s in sets for g in s]
+    assert all(len(s) == K for s in sets) and all(g.numel() == D and g.dtype == flat[0].dtype for g in flat)
+    ptrs = _ptr_array(flat)
+    ordp = _order_array(order)
+    _check(lib().gaf_filter_accumulate_repeat(
+        int(repeats), len(sets), ctypes.cast(ptrs, ctypes.c_void_p), K, D, _dtype_code(flat[0]), float(tau),
+        ordp and ctypes.cast(ordp, ctypes.c_void_p), macro_out.data_ptr(), mask_out.data_ptr(),
+        dist_out.data_ptr(), count_out.data_ptr(), workspace.data_ptr(), workspace.numel(), int(schedule),
+        _stream()), "gaf_filter_accumulate_repeat")
+
+
 def gaf_filter_accumulate_any_seed(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,
                                    macro_out: Optional[torch.Tensor] = None):
     """Order-indifferent variant (end of Section 3.1): every gradient in turn is the seed, ring
@@ -304,3 +325,9 @@ def gaf_last_launch_count() -> int:
 def gaf_last_schedule() -> int:
     """The GAF_SCHED_* value the latest gaf_filter_accumulate call of this thread ran with."""
     return lib().gaf_last_schedule()
+
+
+def gaf_test_set_wait_fault(wait_limit: int, withhold: bool) -> None:
+    """Test hook: poll limit of the kernels' bounded waits and whether the awaited signal is withheld,
+    for the following launches of this thread.  ``(0, False)`` restores normal operation."""
+    _check(lib().gaf_test_set_wait_fault(int(wait_limit), 1 if withhold else 0), "gaf_test_set_wait_fault")

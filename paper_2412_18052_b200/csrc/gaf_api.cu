@@ -2,8 +2,10 @@
 // carve-up and kernel launches.  No device memory is allocated here.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/gaf.h"
 #include "gaf_bucketed.cuh"
@@ -12,6 +14,7 @@
 #include "gaf_gram_panel.cuh"
 #include "gaf_gram_tc.cuh"
 #include "gaf_gramfilter.cuh"
+#include "gaf_host.h"
 #include "gaf_pairwise.cuh"
 #include "gaf_stepwise.cuh"
 #include "gaf_stream.cuh"
@@ -23,7 +26,14 @@ using namespace gaf;
 thread_local int g_launches = 0;
 thread_local int g_schedule = 0;       // what the latest gaf_filter_accumulate resolved AUTO to
 
+// Test hook (gaf_test_set_wait_fault): poll limit and withheld signal for the next launches of this thread.
+thread_local unsigned int g_test_wait_limit = 0;       // 0: the kernels' own limits
+thread_local int g_test_withhold = 0;
+
+constexpr int kMaxDevices = 64;
+
 struct DeviceInfo {
+    int dev = 0;
     int sms = 0;
     int l2_bytes = 0;
     int smem_per_sm = 0;                // shared memory of one SM
@@ -31,19 +41,59 @@ struct DeviceInfo {
     int cooperative = 0;                // cooperative launches supported
 };
 
-// Attributes of the current device (queried per call: a cheap driver lookup).
+// What is worked out once per device and kept for the life of the process: the device's attributes and, per
+// kernel instantiation, its launch plan (occupancy, shared-memory attributes, grid).  A call then costs
+// argument checks and the launch itself: at a million elements the driver queries were a third of the call.
+// Device memory is not involved; the tables are guarded by one mutex on their slow path only.
+std::mutex g_plan_mutex;
+
+// Runs `make(slot)` once per (table slot, device); afterwards the slot is read without the lock.
+template <typename Plan, typename Make>
+int plan_once(Plan &slot, std::atomic<int> &ready, Make &&make) {
+    if (ready.load(std::memory_order_acquire)) return GAF_OK;
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    if (ready.load(std::memory_order_relaxed)) return GAF_OK;
+    if (int rc = make(slot)) return rc;             // nothing is remembered about a failure
+    ready.store(1, std::memory_order_release);
+    return GAF_OK;
+}
+
+struct DeviceSlot { DeviceInfo info; std::atomic<int> ready{0}; };
+DeviceSlot g_devices[kMaxDevices];
+
+// Attributes of the current device.
 bool device_info(DeviceInfo *out) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&out->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&out->l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&out->smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
-        return false;
-    if (cudaDeviceGetAttribute(&out->smem_per_cta_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-        return false;
-    if (cudaDeviceGetAttribute(&out->cooperative, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return false;
-    return out->sms > 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return false;
+    DeviceSlot &slot = g_devices[dev];
+    const int rc = plan_once(slot.info, slot.ready, [dev](DeviceInfo &d) {
+        d.dev = dev;
+        if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GAF_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess) return GAF_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
+            return GAF_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&d.smem_per_cta_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return GAF_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&d.cooperative, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess)
+            return GAF_ERR_CUDA;
+        return d.sms > 0 ? GAF_OK : GAF_ERR_CUDA;
+    });
+    if (rc != GAF_OK) return false;
+    *out = slot.info;
+    return true;
 }
+
+// One slot per device for a kernel instantiation: `static PerDevice<Plan> table;` inside a function template
+// gives every instantiation its own table.
+template <typename Plan>
+struct PerDevice {
+    Plan plan[kMaxDevices];
+    std::atomic<int> ready[kMaxDevices];
+    PerDevice() { for (auto &r : ready) r.store(0, std::memory_order_relaxed); }
+};
+struct DynSmemPlan { int dyn = 0; };    // "the dynamic shared memory limit of this kernel has been raised"
+struct OccPlan { int occ = 1; };
+struct FusedPlan { int occ = 0, park = 0, dyn = 0; };
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t elem_bytes(int dtype) { return dtype == GAF_F32 ? 4 : 2; }
@@ -130,7 +180,8 @@ size_t pairwise_extra_bytes(int K) {
 // Tiled Gram matrix of K gradients (by original index) into the workspace; optional
 // distance matrix.  Two launches.
 int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, float *dist_out,
-                      double *gram_out, unsigned char *base, int sms, cudaStream_t st) {
+                      double *gram_out, unsigned char *base, const DeviceInfo &di, cudaStream_t st) {
+    const int sms = di.sms;
     GramArgs a{};
     for (int i = 0; i < K; ++i) a.g[i] = grads[i];
     a.K = K; a.D = D;
@@ -157,8 +208,18 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         a.slices = int(slices);
         const int dyn = kTcStages * kTcStageBytes + 1024;
         auto kernel = t.Kp == 64 ? gram_tc_kernel<true> : gram_tc_kernel<false>;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
-            return GAF_ERR_CUDA;
+        {
+            static PerDevice<DynSmemPlan> table[2];
+            const int w = t.Kp == 64 ? 1 : 0;
+            if (int rc = plan_once(table[w].plan[di.dev], table[w].ready[di.dev], [&](DynSmemPlan &pl) {
+                    pl.dyn = dyn;
+                    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) == cudaSuccess
+                        ? GAF_OK : GAF_ERR_CUDA;
+                }))
+                return rc;
+        }
+        t.spin_limit = g_test_wait_limit ? g_test_wait_limit : kTcSpinLimit;
+        t.test_extra_arrival = g_test_withhold;
         kernel<<<a.slices, t.Kp == 64 ? kTcThreadsWide : kTcThreads, dyn, st>>>(t);
         ++g_launches;
     } else {
@@ -187,8 +248,19 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
             kernel = shift == 7 ? gram_panel_kernel<__nv_bfloat16, 7, 4>
                    : (shift == 6 ? (wpp == 2 ? gram_panel_kernel<__nv_bfloat16, 6, 2> : gram_panel_kernel<__nv_bfloat16, 6, 1>)
                                  : gram_panel_kernel<__nv_bfloat16, 5, 1>);
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
-            return GAF_ERR_CUDA;
+        {
+            // (the kernel pointer is the key: six instantiations per input type)
+            static PerDevice<DynSmemPlan> table[2][4];
+            const int v = shift == 7 ? 0 : (shift == 6 ? (wpp == 2 ? 1 : 2) : 3);
+            auto &tb = table[dtype == GAF_F32 ? 0 : 1][v];
+            if (int rc = plan_once(tb.plan[di.dev], tb.ready[di.dev], [&](DynSmemPlan &pl) {
+                    // the largest panel this instantiation is ever launched with
+                    pl.dyn = kPanelStages * (shift == 7 ? 2 : (shift == 6 ? 4 : 8)) * 8 * row_bytes;
+                    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.dyn) == cudaSuccess
+                        ? GAF_OK : GAF_ERR_CUDA;
+                }))
+                return rc;
+        }
         const int64_t chunk_elems = row_bytes / int64_t(elem_bytes(dtype));
         const int64_t work = (D + chunk_elems - 1) / chunk_elems;
         int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;      // one CTA per SM
@@ -208,13 +280,18 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
 }
 
 template <typename T, int KT>
-int launch_gram_small_kt(const GramSmallArgs &a, int sms, cudaStream_t st) {
-    int occ = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gram_small_kernel<T, KT>, kGsThreads, 0) !=
-        cudaSuccess || occ < 1)
-        occ = 1;
-    if (occ > 2) occ = 2;
-    int64_t grid = int64_t(sms) * occ;
+int launch_gram_small_kt(const GramSmallArgs &a, const DeviceInfo &di, cudaStream_t st) {
+    static PerDevice<OccPlan> table;
+    plan_once(table.plan[di.dev], table.ready[di.dev], [](OccPlan &pl) {
+        int occ = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gram_small_kernel<T, KT>, kGsThreads, 0) !=
+            cudaSuccess || occ < 1)
+            occ = 1;
+        pl.occ = occ > 2 ? 2 : occ;
+        return GAF_OK;
+    });
+    const int occ = table.plan[di.dev].occ;
+    int64_t grid = int64_t(di.sms) * occ;
     if (grid > kGsMaxCtas) grid = kGsMaxCtas;
     const int64_t work = (a.D / GsVec<T>::N + kGsThreads - 1) / kGsThreads;
     if (grid > work) grid = work;
@@ -225,15 +302,15 @@ int launch_gram_small_kt(const GramSmallArgs &a, int sms, cudaStream_t st) {
 }
 
 template <typename T>
-int launch_gram_small(const GramSmallArgs &a, int K, int sms, cudaStream_t st) {
+int launch_gram_small(const GramSmallArgs &a, int K, const DeviceInfo &di, cudaStream_t st) {
     switch (K) {
-        case 2: return launch_gram_small_kt<T, 2>(a, sms, st);
-        case 3: return launch_gram_small_kt<T, 3>(a, sms, st);
-        case 4: return launch_gram_small_kt<T, 4>(a, sms, st);
-        case 5: return launch_gram_small_kt<T, 5>(a, sms, st);
-        case 6: return launch_gram_small_kt<T, 6>(a, sms, st);
-        case 7: return launch_gram_small_kt<T, 7>(a, sms, st);
-        case 8: return launch_gram_small_kt<T, 8>(a, sms, st);
+        case 2: return launch_gram_small_kt<T, 2>(a, di, st);
+        case 3: return launch_gram_small_kt<T, 3>(a, di, st);
+        case 4: return launch_gram_small_kt<T, 4>(a, di, st);
+        case 5: return launch_gram_small_kt<T, 5>(a, di, st);
+        case 6: return launch_gram_small_kt<T, 6>(a, di, st);
+        case 7: return launch_gram_small_kt<T, 7>(a, di, st);
+        case 8: return launch_gram_small_kt<T, 8>(a, di, st);
         default: return GAF_ERR_ARG;
     }
 }
@@ -254,45 +331,55 @@ constexpr int64_t kFusedMaxInputBytesF32 = int64_t(512) << 20;
 template <typename T, int KT>
 int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st) {
     auto kernel = gram_fused_kernel<T, KT>;
-    // CTAs per SM by registers alone, then as many parked rounds as shared memory allows
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kGsThreads, 0) != cudaSuccess || occ < 1)
-        return GAF_ERR_UNSUPPORTED;
-    if (occ > 2) occ = 2;
-    cudaFuncAttributes fa{};
-    if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return GAF_ERR_CUDA;
-    const int round_bytes = KT * kGsThreads * 16;
-    int64_t budget = di.smem_per_sm / occ - 1024 - int64_t(fa.sharedSizeBytes);
-    if (budget > di.smem_per_cta_max - int64_t(fa.sharedSizeBytes)) budget = di.smem_per_cta_max - int64_t(fa.sharedSizeBytes);
-    if (budget > kParkBytesPerSm / occ) budget = kParkBytesPerSm / occ;
-    const int park = budget > 0 ? int(budget / round_bytes) : 0;
-    const int dyn = park * round_bytes;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
-        return GAF_ERR_CUDA;
-    {
-        // shared memory share of the L1/shared array: what the CTAs of one SM need, no more (the rest is L1)
-        int pct = int((int64_t(dyn + fa.sharedSizeBytes + 1024) * occ * 100 + di.smem_per_sm - 1) / di.smem_per_sm);
-        if (pct > 100) pct = 100;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, pct) != cudaSuccess)
-            return GAF_ERR_CUDA;
-    }
-    int occ2 = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ2, kernel, kGsThreads, dyn) != cudaSuccess || occ2 < 1)
-        return GAF_ERR_UNSUPPORTED;
-    if (occ2 < occ) occ = occ2;
-    int64_t grid = int64_t(di.sms) * occ;
+    // The plan of this instantiation on this device: CTAs per SM by registers alone, then as many parked
+    // rounds as shared memory allows; the kernel's shared-memory attributes are set on the way.
+    static PerDevice<FusedPlan> table;
+    if (int rc = plan_once(table.plan[di.dev], table.ready[di.dev], [&](FusedPlan &pl) {
+            int occ = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kGsThreads, 0) != cudaSuccess || occ < 1)
+                return GAF_ERR_UNSUPPORTED;
+            if (occ > 2) occ = 2;
+            cudaFuncAttributes fa{};
+            if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return GAF_ERR_CUDA;
+            const int round_bytes = KT * kGsThreads * 16;
+            int64_t budget = di.smem_per_sm / occ - 1024 - int64_t(fa.sharedSizeBytes);
+            if (budget > di.smem_per_cta_max - int64_t(fa.sharedSizeBytes))
+                budget = di.smem_per_cta_max - int64_t(fa.sharedSizeBytes);
+            if (budget > kParkBytesPerSm / occ) budget = kParkBytesPerSm / occ;
+            const int park = budget > 0 ? int(budget / round_bytes) : 0;
+            const int dyn = park * round_bytes;
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) != cudaSuccess)
+                return GAF_ERR_CUDA;
+            // shared memory share of the L1/shared array: what the CTAs of one SM need, no more (the rest is L1)
+            int pct = int((int64_t(dyn + fa.sharedSizeBytes + 1024) * occ * 100 + di.smem_per_sm - 1) / di.smem_per_sm);
+            if (pct > 100) pct = 100;
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, pct) != cudaSuccess)
+                return GAF_ERR_CUDA;
+            int occ2 = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ2, kernel, kGsThreads, dyn) != cudaSuccess || occ2 < 1)
+                return GAF_ERR_UNSUPPORTED;
+            pl.occ = occ2 < occ ? occ2 : occ;
+            pl.park = park;
+            pl.dyn = dyn;
+            return GAF_OK;
+        }))
+        return rc;
+    const FusedPlan &pl = table.plan[di.dev];
+    int64_t grid = int64_t(di.sms) * pl.occ;
     if (grid > kGsMaxCtas) grid = kGsMaxCtas;
     const int64_t work = (a.D / FusedVec<T>::N + kGsThreads - 1) / kGsThreads;
     if (grid > work) grid = work;
     if (grid < 1) grid = 1;
-    a.park_rounds = park;
+    a.park_rounds = pl.park;
+    a.spin_limit = g_test_wait_limit ? g_test_wait_limit : kFusedSpinLimit;
+    a.test_withhold = g_test_withhold;
     // the last stretch is asked to stay in L2 for the second pass
     const int64_t per_elem = int64_t(KT) * int64_t(sizeof(T));
     const int64_t keep_elems = int64_t(di.l2_bytes) * kKeepL2Pct / 100 / per_elem;
     a.keep_from = a.D > keep_elems ? a.D - keep_elems : 0;
     void *params[] = {&a};
     const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kernel), dim3(int(grid)),
-                                                        dim3(kGsThreads), params, size_t(dyn), st);
+                                                        dim3(kGsThreads), params, size_t(pl.dyn), st);
     if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     ++g_launches;
     return GAF_OK;
@@ -356,9 +443,9 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
         a.gram = gram_by_step;
         a.replay = r;
         a.ring = ring;
-        if (int rc = launch_gram_small<T>(a, K, sms, st)) return rc;
+        if (int rc = launch_gram_small<T>(a, K, di, st)) return rc;
     } else {
-        if (int rc = launch_gram_tiles(g, K, D, dtype, nullptr, nullptr, base, sms, st)) return rc;
+        if (int rc = launch_gram_tiles(g, K, D, dtype, nullptr, nullptr, base, di, st)) return rc;
         if (seed_out) gram_ring_replay_kernel<<<1, GAF_MAX_K, 0, st>>>(ring, gram_by_index);
         else gram_replay_kernel<<<1, 256, 0, st>>>(r, gram_by_index, gram_by_step);
         ++g_launches;
@@ -452,6 +539,8 @@ int launch_bucket_gram(const BucketGramArgs &a, const BucketTable &bt, int K, in
 
 }  // namespace
 
+void gaf::set_last_launch_count(int launches) { g_launches = launches; }
+
 extern "C" {
 
 const char *gaf_error_string(int code) {
@@ -471,6 +560,12 @@ const char *gaf_error_string(int code) {
 
 int gaf_last_launch_count(void) { return g_launches; }
 int gaf_last_schedule(void) { return g_schedule; }
+
+int gaf_test_set_wait_fault(unsigned int wait_limit, int withhold) {
+    g_test_wait_limit = wait_limit;
+    g_test_withhold = withhold ? 1 : 0;
+    return GAF_OK;
+}
 
 int gaf_workspace_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {
     if (!bytes_out || K < 1 || K > GAF_MAX_K || D < 0) return GAF_ERR_ARG;
@@ -565,6 +660,24 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
                                  ctl, partials, di.sms, st)
         : launch_stepwise<__nv_bfloat16>(grads, K, D, tau, ord, macro_out, mask_out, dist_out,
                                          count_out, ctl, partials, di.sms, st);
+}
+
+int gaf_filter_accumulate_repeat(int repeats, int n_sets, const void *const *grads, int K, int64_t D,
+                                 int dtype, double tau, const int32_t *order, float *macro_out,
+                                 uint8_t *mask_out, float *dist_out, int32_t *count_out, void *workspace,
+                                 size_t workspace_bytes, int schedule, void *cuda_stream) {
+    g_launches = 0;
+    if (repeats < 0 || n_sets < 1 || !grads || K < 1 || K > GAF_MAX_K) return GAF_ERR_ARG;
+    int launches = 0;
+    for (int r = 0; r < repeats; ++r) {
+        const int rc = gaf_filter_accumulate(grads + size_t(r % n_sets) * K, K, D, dtype, tau, order, macro_out,
+                                             mask_out, dist_out, count_out, workspace, workspace_bytes,
+                                             schedule, cuda_stream);
+        if (rc != GAF_OK) return rc;
+        launches += g_launches;
+    }
+    g_launches = launches;
+    return GAF_OK;
 }
 
 int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, int dtype, double tau,
@@ -832,10 +945,10 @@ int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype, 
         a.replay.ctl = reinterpret_cast<Control *>(base);
         a.pair_dist_out = dist_out;
         a.pair_gram_out = gram_out;
-        return dtype == GAF_F32 ? launch_gram_small<float>(a, K, di.sms, st)
-                                : launch_gram_small<__nv_bfloat16>(a, K, di.sms, st);
+        return dtype == GAF_F32 ? launch_gram_small<float>(a, K, di, st)
+                                : launch_gram_small<__nv_bfloat16>(a, K, di, st);
     }
-    return launch_gram_tiles(grads, K, D, dtype, dist_out, gram_out, base, di.sms, st);
+    return launch_gram_tiles(grads, K, D, dtype, dist_out, gram_out, base, di, st);
 }
 
 int gaf_read_status(const void *workspace, void *cuda_stream, int *status_out) {

@@ -95,7 +95,6 @@ bucket_gram_kernel(const __grid_constant__ BucketGramArgs a, const __grid_consta
                 const int64_t q = qw + lane;
                 if (q < n_vec) {
                     float x[KT][N];
-#pragma unroll
                     const uint64_t pol = (s0 + q * N >= hi - a.keep_elems) ? pol_last : pol_first;
 #pragma unroll
                     for (int r = 0; r < KT; ++r) GsVec<T>::load(row[r], s0 + q * N, pol, x[r]);
@@ -217,7 +216,7 @@ bucket_walk_kernel(const __grid_constant__ BucketWalkArgs a, const __grid_consta
     if (threadIdx.x == 0) {
         int status = 0, count = 1;
         unsigned long long bits = 1ull;
-        double na = sgram[0];
+        double na = sgram[0], norm_sq = sgram[0];
         uint8_t *mask = a.mask_out + (size_t)b * K;
         float *dist = a.dist_out ? a.dist_out + (size_t)b * K : nullptr;
         mask[a.idx[0]] = 1;
@@ -231,7 +230,10 @@ bucket_walk_kernel(const __grid_constant__ BucketWalkArgs a, const __grid_consta
             const int accept = (d <= a.tau) ? 1 : 0;
             mask[a.idx[t]] = (uint8_t)accept;
             if (dist) dist[a.idx[t]] = (float)d;
-            if (accept) { bits |= 1ull << t; na = na + 2.0 * p + ng; ++count; }
+            if (accept) {
+                bits |= 1ull << t; na = na + 2.0 * p + ng; norm_sq += ng; ++count;
+                status |= ill_conditioned(count, norm_sq, na);
+            }
         }
         a.bits[b] = bits;
         a.count_out[b] = count;

@@ -27,6 +27,7 @@ struct Control {
     double sums[GAF_MAX_K][3];          // by step t: {g_i.g, |g|^2, |g_i|^2}
     float stream_dist[GAF_MAX_K];       // streaming form: distance of arrival t
     uint8_t stream_mask[GAF_MAX_K];     // streaming form: decision of arrival t
+    double norm_sq_sum;                 // stepwise and streaming forms: sum of |g_i|^2 over the accepted gradients
     // One-launch Gram-first schedule: the word the waiting CTAs poll, alone in its cache line.
     // Bits 16..31 call generation, 8..15 winning seed + 1 (0: no any-seed walk), 0..7 accept bits.
     alignas(128) unsigned int fused_word;
@@ -201,6 +202,19 @@ __device__ __forceinline__ double cosine_distance(double p, double na, double ng
     }
     if (!(isfinite(p) && isfinite(na) && isfinite(ng))) *status |= GAF_STATUS_NONFINITE;
     return 1.0 - cosv;
+}
+
+// Conditioning of a running sum g of c accepted gradients.  Every schedule forms |g|^2 (and g itself)
+// from binary32-rounded quantities, so its relative error is about 6e-8 kappa with
+//     kappa = c * sum_i |g_i|^2 / |g|^2   (>= (sum_i |g_i|)^2 / |g|^2 >= 1),
+// which is at most c while no accepted gradient points against the sum (tau <= 1), and grows without
+// bound when accepted gradients nearly cancel (possible only with tau > 1).  Beyond kIllKappa the
+// distance tolerance of 1e-5 (6e-8 kappa > 1e-5) and the 1e-6 of the binary32 macro-gradient are no
+// longer guaranteed: the call says so with GAF_STATUS_ILL_CONDITIONED.  `norm_sq_sum` = sum_i |g_i|^2
+// and `na` = |g|^2, both for the sum AFTER an accept.
+constexpr double kIllKappa = 167.0;
+__device__ __forceinline__ int ill_conditioned(int c, double norm_sq_sum, double na) {
+    return ((double)c * norm_sq_sum > kIllKappa * na) ? GAF_STATUS_ILL_CONDITIONED : 0;
 }
 
 }  // namespace gaf

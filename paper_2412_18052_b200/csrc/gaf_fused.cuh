@@ -38,6 +38,9 @@ struct GramFusedArgs {
     float *out;                             // D floats
     ReplayArgs replay;                      // used when ring.K == 0
     RingArgs ring;                          // any-seed mode when ring.K > 0
+    unsigned int spin_limit;                // polls a waiting CTA makes before it gives up
+    int test_withhold;                      // test hook, normally 0: the deciding CTA does not publish the
+                                            // decision word, so that every other CTA's wait runs out
 };
 
 // The polled word carries its own payload, so no ordering with other memory is needed.
@@ -198,7 +201,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
         auto notice = [&](int seed, unsigned long long bits) {
             const unsigned int word = ((gen0 + 1u) << 16) | ((unsigned int)(seed + 1) << 8) | (unsigned int)(bits & 0xFFull);
             decided = word;
-            st_relaxed_u32(&ctl->fused_word, word);
+            if (!a.test_withhold) st_relaxed_u32(&ctl->fused_word, word);
         };
         if (a.ring.K > 0) {
             __shared__ RingTable<KT> ring_table;
@@ -215,7 +218,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
             unsigned int polls = 0;
             while (((word = ld_relaxed_u32(&ctl->fused_word)) >> 16) == gen0) {
                 __nanosleep(40);
-                if (++polls > kFusedSpinLimit) { ok = false; break; }
+                if (++polls > a.spin_limit) { ok = false; break; }
             }
         }
         if (!ok) {

@@ -64,6 +64,9 @@ struct GramTcArgs {
     double *partials;       // [tile pair][slice][64]
     int tiles;              // ceil(K / 8)
     Control *ctl;
+    unsigned int spin_limit;    // attempts (of up to ~2 us each) a wait makes before it gives up
+    int test_extra_arrival;     // test hook, normally 0: the first tile's barrier expects one arrival more
+                                // than will ever come, so that every wait of the pipeline runs out
 };
 
 // ----------------------------------------------------------------- PTX --------
@@ -93,8 +96,9 @@ __device__ __forceinline__ bool tc_mbar_try(uint64_t *bar, uint32_t parity, uint
     return ok != 0;
 }
 // Bounded wait: false when the limit ran out or another thread already gave up.
-__device__ __forceinline__ bool tc_mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    for (unsigned int spin = 0; spin < kTcSpinLimit; ++spin) {
+__device__ __forceinline__ bool tc_mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                             unsigned int limit) {
+    for (unsigned int spin = 0; spin < limit; ++spin) {
         if (tc_mbar_try(bar, parity, 2000u)) return true;
         if (*abort_flag) return false;
     }
@@ -104,9 +108,10 @@ __device__ __forceinline__ bool tc_mbar_wait(uint64_t *bar, uint32_t parity, vol
 // The same for a whole warp: one lane polls (32 lanes polling one mbarrier are 32 serialised
 // shared-memory operations per round), the others learn the outcome through the shuffle,
 // which also orders their later accesses after the polling lane's acquire.
-__device__ __forceinline__ bool tc_mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool tc_mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                                  unsigned int limit) {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = tc_mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = tc_mbar_wait(bar, parity, abort_flag, limit) ? 1 : 0;
     return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 __device__ __forceinline__ void tc_cp_async16(uint32_t dst_smem, const void *src) {
@@ -172,6 +177,7 @@ struct GramTcShared {
     uint64_t empty[kTcStages];      // MMA -> loaders: tile consumed
     uint64_t acc_full[2];           // MMA -> epilogue: accumulator buffer complete
     uint64_t acc_empty[2];          // epilogue -> MMA: accumulator buffer read out
+    uint64_t drained;               // MMA thread, after a wait gave up: the MMAs it had issued are complete
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -203,13 +209,15 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
-            tc_mbar_init(&sh.full[s], kTcLoaders);       // every loader thread arrives
+            // every loader thread arrives
+            tc_mbar_init(&sh.full[s], kTcLoaders + ((s == 0 && a.test_extra_arrival) ? 1 : 0));
             tc_mbar_init(&sh.empty[s], 1);               // one commit
         }
         for (int b = 0; b < 2; ++b) {
             tc_mbar_init(&sh.acc_full[b], 1);
             tc_mbar_init(&sh.acc_empty[b], WIDE ? 256 : 128);    // every epilogue thread arrives
         }
+        tc_mbar_init(&sh.drained, 1);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (blockIdx.x == 0) a.ctl->status = 0;          // first kernel of the operation
@@ -271,7 +279,7 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
         for (int it = 0; it < n_tiles; ++it) {
             const int s = it % kTcStages;
             if (it >= kTcStages &&
-                !tc_mbar_wait_warp(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag))
+                !tc_mbar_wait_warp(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag, a.spin_limit))
                 break;
             const int64_t elem0 = (blockIdx.x + it * G) * unit;       // first element of the tile, per gradient
             const int64_t byte0 = elem0 * 2;
@@ -304,9 +312,12 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
                 const bool first_of_block = (it % kTcDrain) == 0;
                 if (first_of_block && blk >= 2) {
                     // the epilogue must have read this buffer's previous contents
-                    if (!tc_mbar_wait(&sh.acc_empty[buf], (uint32_t)((blk / 2 - 1) & 1), &sh.abort_flag)) break;
+                    if (!tc_mbar_wait(&sh.acc_empty[buf], (uint32_t)((blk / 2 - 1) & 1), &sh.abort_flag, a.spin_limit)) break;
                 }
-                if (!tc_mbar_wait(&sh.full[s], (uint32_t)((it / kTcStages) & 1), &sh.abort_flag)) break;
+                if (!tc_mbar_wait(&sh.full[s], (uint32_t)((it / kTcStages) & 1), &sh.abort_flag, a.spin_limit)) break;
+                // the tile was written by cp.async (generic proxy) and is read by the MMA through the
+                // asynchronous proxy: order the two before the first MMA of the tile
+                tc_fence_async_smem();
                 tc_fence_after_sync();
 #pragma unroll
                 for (int b = 0; b < kTcSub; ++b) {
@@ -321,6 +332,12 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
                 tc_commit(&sh.empty[s]);
                 if ((it % kTcDrain) == kTcDrain - 1 || it == n_tiles - 1) tc_commit(&sh.acc_full[buf]);
             }
+            // Tensor memory must not be freed under MMAs still in flight (a wait that gave up, here or in
+            // another warp, skips the handshakes that normally guarantee it): one more commit arrives when
+            // everything issued so far has completed.  Bounded like every wait; it ignores the abort flag.
+            tc_commit(&sh.drained);
+            for (unsigned int spin = 0; spin < a.spin_limit; ++spin)
+                if (tc_mbar_try(&sh.drained, 0u, 2000u)) break;
         }
         __syncwarp();
     } else {
@@ -328,7 +345,7 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
         for (int blk = 0; blk < n_blocks; ++blk) {
             const int buf = blk & 1;
             // (warp-uniform outcome: the load below needs the whole warp)
-            if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag)) break;
+            if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag, a.spin_limit)) break;
             tc_fence_after_sync();
             uint32_t r[32];
             tc_tmem_ld32(tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128 + epi_col0), r);

@@ -46,6 +46,7 @@ __device__ __forceinline__ unsigned long long replay_on_gram(const ReplayArgs &r
     int status = 0, count = 1;
     unsigned long long bits = 1ull;         // step 0 is the seed
     double na = gram[0];                    // |g|^2 of the running sum
+    double norm_sq = gram[0];               // sum of |g_i|^2 over the accepted gradients
     if (publish) {
         c->decision[0] = 1;
         r.mask_out[r.idx[0]] = 1;
@@ -67,14 +68,17 @@ __device__ __forceinline__ unsigned long long replay_on_gram(const ReplayArgs &r
         if (accept) {
             bits |= 1ull << t;
             na = na + 2.0 * p + ng;         // |g + g_t|^2
+            norm_sq += ng;
             ++count;
+            status |= ill_conditioned(count, norm_sq, na);
         }
     }
     if (publish) {
         c->accept_bits = bits;
         c->ring_seed = -1;
         c->count = count;
-        c->status = status;
+        // (OR, not store: an earlier kernel of the operation may have raised a bit; the first kernel cleared the word)
+        if (status) atomicOr(&c->status, status);
         *r.count_out = count;
     }
     return bits;
@@ -108,7 +112,8 @@ __device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, con
         // Branch-free (neighbouring lanes hold different cases): a gradient that is not in the case
         // contributes an added 0.0, which leaves a binary64 sum unchanged, and its update of |g|^2
         // is computed and dropped.
-        double na = gram[0];
+        double na = gram[0], norm_sq = gram[0];
+        int cnt = 1;
 #pragma unroll
         for (int u = 1; u < K - 1; ++u) {
             double pu = 0.0;
@@ -116,14 +121,20 @@ __device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, con
             for (int v = 0; v < u; ++v) pu += in(v) ? gram[v * K + u] : 0.0;
             const double grown = na + 2.0 * pu + gram[u * K + u];
             na = in(u) ? grown : na;
+            norm_sq += in(u) ? gram[u * K + u] : 0.0;
+            cnt += in(u) ? 1 : 0;
         }
         double p = 0.0;
 #pragma unroll
         for (int v = 0; v < K - 1; ++v) p += (v < t && in(v)) ? gram[v * K + t] : 0.0;
         int status = 0;
-        const double d = cosine_distance(p, na, gram[t * K + t], &status);
+        const double ng = gram[t * K + t];
+        const double d = cosine_distance(p, na, ng, &status);
+        const int accept = (d <= r.tau) ? 1 : 0;
+        // the sum this case would leave behind, if it accepts
+        status |= accept ? ill_conditioned(cnt + 1, norm_sq + ng, na + 2.0 * p + ng) : 0;
         tb.d[tid] = d; tb.p[tid] = p; tb.na[tid] = na;
-        tb.accept[tid] = (d <= r.tau) ? 1 : 0;
+        tb.accept[tid] = (unsigned char)accept;
         tb.status[tid] = (unsigned char)status;
     }
     __syncthreads();
@@ -153,7 +164,7 @@ __device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, con
         c->accept_bits = bits;
         c->ring_seed = -1;
         c->count = count;
-        c->status = status;
+        if (status) atomicOr(&c->status, status);
         *r.count_out = count;
         __threadfence();
     }
@@ -180,7 +191,7 @@ __device__ __forceinline__ void ring_walk_one_seed(const RingArgs &r, const vola
     const int K = r.K;
     unsigned long long bits = 1ull << s;    // bit i set = gradient i (original index) accepted
     int count = 1, status = 0;
-    double na = gram[(size_t)s * K + s];
+    double na = gram[(size_t)s * K + s], norm_sq = na;
     if (dist_by_index) dist_by_index[s] = 0.0f;
     for (int t = 1; t < K; ++t) {
         const int i = (s + t) % K;
@@ -195,7 +206,9 @@ __device__ __forceinline__ void ring_walk_one_seed(const RingArgs &r, const vola
         if (d <= r.tau) {
             bits |= 1ull << i;
             na = na + 2.0 * p + ng;
+            norm_sq += ng;
             ++count;
+            status |= ill_conditioned(count, norm_sq, na);
         }
     }
     count_out = count; bits_out = bits; status_out = status;
@@ -233,7 +246,7 @@ __device__ __forceinline__ void ring_replay_on_gram(const RingArgs &r, const vol
         ctl->accept_bits = b;
         ctl->ring_seed = best;
         ctl->count = c;
-        ctl->status = st;
+        if (st) atomicOr(&ctl->status, st);
         *r.count_out = c;
         *r.seed_out = best;
         __threadfence();
@@ -264,22 +277,29 @@ __device__ __forceinline__ void ring_replay_parallel(const RingArgs &r, const do
         const unsigned int m = (unsigned int)(cs + 1) - (1u << (t - 1));
         auto in = [&](int v) { return v == 0 || ((m >> (v - 1)) & 1u); };
         auto gi = [&](int v) { const int i = s + v; return i >= K ? i - K : i; };      // gradient of step v
-        double na = gram[s * K + s];
+        double na = gram[s * K + s], norm_sq = na;
+        int cnt = 1;
 #pragma unroll
         for (int u = 1; u < K - 1; ++u) {
             double pu = 0.0;
 #pragma unroll
             for (int v = 0; v < u; ++v) pu += in(v) ? gram[gi(v) * K + gi(u)] : 0.0;
-            const double grown = na + 2.0 * pu + gram[gi(u) * K + gi(u)];
+            const double guu = gram[gi(u) * K + gi(u)];
+            const double grown = na + 2.0 * pu + guu;
             na = in(u) ? grown : na;
+            norm_sq += in(u) ? guu : 0.0;
+            cnt += in(u) ? 1 : 0;
         }
         double p = 0.0;
 #pragma unroll
         for (int v = 0; v < K - 1; ++v) p += (v < t && in(v)) ? gram[gi(v) * K + gi(t)] : 0.0;
         int status = 0;
-        const double d = cosine_distance(p, na, gram[gi(t) * K + gi(t)], &status);
+        const double ng = gram[gi(t) * K + gi(t)];
+        const double d = cosine_distance(p, na, ng, &status);
+        const int accept = (d <= r.tau) ? 1 : 0;
+        status |= accept ? ill_conditioned(cnt + 1, norm_sq + ng, na + 2.0 * p + ng) : 0;
         tb.d[idx] = (float)d;
-        tb.accept[idx] = (d <= r.tau) ? 1 : 0;
+        tb.accept[idx] = (unsigned char)accept;
         tb.status[idx] = (unsigned char)status;
     }
     __syncthreads();
@@ -318,7 +338,7 @@ __device__ __forceinline__ void ring_replay_parallel(const RingArgs &r, const do
         ctl->accept_bits = bits;
         ctl->ring_seed = best;
         ctl->count = tb.count[best];
-        ctl->status = status;
+        if (status) atomicOr(&ctl->status, status);
         *r.count_out = tb.count[best];
         *r.seed_out = best;
         __threadfence();

@@ -17,6 +17,7 @@
 #include <mutex>
 
 #include "../../include/gaf.h"
+#include "gaf_host.h"
 #include "gaf_stepwise.cuh"
 
 namespace {
@@ -56,6 +57,7 @@ int static_scratch(void **out) {
 
 extern "C" int gaf_cosdist_static(const void *x, const void *y, int64_t D, int dtype,
                                   float *dist_out, double *stats_out, void *cuda_stream) {
+    set_last_launch_count(0);
     if (D < 0 || ((!x || !y) && D > 0) || !dist_out) return GAF_ERR_ARG;
     if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
     if (D > GAF_STATIC_MAX_D) return GAF_ERR_TOO_LARGE;
@@ -87,5 +89,6 @@ extern "C" int gaf_cosdist_static(const void *x, const void *y, int64_t D, int d
               reinterpret_cast<double *>(base + kStaticControlBytes), dist_out, stats_out};
     if (dtype == GAF_F32) cosdist_kernel<float><<<int(grid), kStepThreads, 0, st>>>(a);
     else cosdist_kernel<__nv_bfloat16><<<int(grid), kStepThreads, 0, st>>>(a);
+    set_last_launch_count(1);
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }

@@ -52,6 +52,13 @@ __device__ __forceinline__ void finalize_step(const StepArgs &a, Sums3 mine, int
         c->decision[step_next] = accept;
         c->sums[step_next][0] = tot.p; c->sums[step_next][1] = tot.na; c->sums[step_next][2] = tot.ng;
         c->count += accept;
+        if (step_next == 1) c->norm_sq_sum = tot.na;        // the running sum is still the seed alone
+        if (accept) {
+            // conditioning of the sum this accept leaves behind: |g + g_i|^2 from the three sums
+            // (c->count and c->norm_sq_sum are touched by the deciding thread of each launch only)
+            c->norm_sq_sum += tot.ng;
+            status |= ill_conditioned(c->count, c->norm_sq_sum, tot.na + 2.0 * tot.p + tot.ng);
+        }
         if (status) atomicOr(&c->status, status);
         a.mask_out[a.i_next] = (uint8_t)accept;
         if (a.dist_out) a.dist_out[a.i_next] = (float)d;

@@ -71,6 +71,11 @@ __global__ void __launch_bounds__(kStreamThreads, 2) stream_test_kernel(StreamAr
         c->stream_mask[a.t] = (uint8_t)accept;
         c->stream_dist[a.t] = (float)d;
         c->count += accept;
+        if (a.t == 1) c->norm_sq_sum = tot.na;              // the running sum is still the seed alone
+        if (accept) {
+            c->norm_sq_sum += tot.ng;
+            status |= ill_conditioned(c->count, c->norm_sq_sum, tot.na + 2.0 * tot.p + tot.ng);
+        }
         if (status) atomicOr(&c->status, status);
         __threadfence();
     }

@@ -65,9 +65,20 @@ def oracle_with_replay(np_grads, tau, order, gpu_mask):
 
 def check_filter(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,
                  order: Optional[Sequence[int]] = None, schedule: int = 0,
-                 np_grads=None, expect_status: Optional[int] = 0):
+                 np_grads=None, expect_status: Optional[int] = 0, allow_ill_conditioned: bool = False):
     """Run gaf_filter_accumulate on the GPU and compare everything with the oracle.
-    Returns a dict of the measured errors."""
+    Returns a dict of the measured errors.  With `allow_ill_conditioned` a comparison that fails is
+    forgiven when (and only when) the library itself raised GAF_STATUS_ILL_CONDITIONED for the call:
+    the accepted gradients nearly cancelled and the library said that its tolerances do not hold."""
+    try:
+        return _check_filter(grads, tau, workspace, order, schedule, np_grads, expect_status)
+    except AssertionError:
+        if allow_ill_conditioned and (gaf.gaf_read_status(workspace) & gaf.GAF_STATUS_ILL_CONDITIONED):
+            return {"ill_conditioned": True}
+        raise
+
+
+def _check_filter(grads, tau, workspace, order, schedule, np_grads, expect_status):
     K, D = len(grads), grads[0].numel()
     dev = grads[0].device
     # guard bands around every output catch out-of-bounds writes
@@ -135,11 +146,24 @@ def check_pairwise(grads: Sequence[torch.Tensor], workspace: torch.Tensor):
     return err
 
 
-def check_any_seed(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor):
+def check_any_seed(grads: Sequence[torch.Tensor], tau: float, workspace: torch.Tensor,
+                   allow_ill_conditioned: bool = False):
     """gaf_filter_accumulate_any_seed against the oracle: the winning seed, and for that
-    seed everything check_filter checks (ring order starting at the seed)."""
+    seed everything check_filter checks (ring order starting at the seed).  `allow_ill_conditioned`
+    as in check_filter."""
     K = len(grads)
     macro, mask, dist, count, seed = gaf.gaf_filter_accumulate_any_seed(grads, tau, workspace)
+    status = gaf.gaf_read_status(workspace)
+    try:
+        return _check_any_seed(grads, tau, workspace, macro, mask, dist, count, seed)
+    except AssertionError:
+        if allow_ill_conditioned and (status & gaf.GAF_STATUS_ILL_CONDITIONED):
+            return {"ill_conditioned": True}
+        raise
+
+
+def _check_any_seed(grads, tau, workspace, macro, mask, dist, count, seed):
+    K = len(grads)
     np_grads = [as_numpy_bits(g) for g in grads]
     want, want_seed, counts = orc.filter_any_seed(np_grads, tau)
     g_seed = int(seed.cpu().item())

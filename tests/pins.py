@@ -420,6 +420,33 @@ def pin_bucketed_variant():
     assert len(seen) >= 2                           # buckets really decide on their own
 
 
+def pin_all_cores_form_equals_single_thread():
+    """The several-threads form of the filter (the benchmark's all-cores CPU baseline) is the same
+    computation: identical masks and counts, distances and outputs equal to 1e-12 (only the order
+    in which the chunk sums are combined differs), for every thread count including more threads
+    than elements, both element types, an explicit order, and the tau = 2 / reject-all pins."""
+    rng = np.random.RandomState(31)
+    for K, D, dtype in ((4, 10_007, np.float32), (5, 1_001, np.uint16), (3, 5, np.float32), (1, 40, np.float32)):
+        if dtype == np.float32:
+            grads = [rng.randn(D).astype(np.float32) + 0.6 * (i % 2) for i in range(K)]
+        else:
+            grads = [(rng.randn(D).astype(np.float32) + 0.5).view(np.uint32).__rshift__(16).astype(np.uint16)
+                     for _ in range(K)]
+        order = [int(x) for x in rng.permutation(K)]
+        for tau in (0.9, 1.0, 2.0, -1.0):
+            want = orc.filter_accumulate(grads, tau, order=order)
+            for n_threads in (1, 2, 3, 7, 16):
+                got = orc.filter_accumulate_all_cores(grads, tau, order=order, n_threads=n_threads)
+                assert got.mask.tolist() == want.mask.tolist() and got.count == want.count
+                assert np.max(np.abs(got.dist - want.dist)) <= 1e-12
+                scale = np.max(np.abs(want.out)) + 1e-300
+                assert np.max(np.abs(got.out - want.out)) <= 1e-12 * scale
+    # tau = 2 is the plain mean of Eq. 2, also through this route
+    grads = [rng.randn(999).astype(np.float32) for _ in range(4)]
+    got = orc.filter_accumulate_all_cores(grads, 2.0, n_threads=4)
+    assert np.allclose(got.out, np.mean(np.stack(grads).astype(np.float64), axis=0), rtol=0, atol=1e-15)
+
+
 ALL_PINS = [
     pin_stated_values,
     pin_figure2_angles,
@@ -438,4 +465,5 @@ ALL_PINS = [
     pin_closed_form_mixture,
     pin_any_seed_variant,
     pin_bucketed_variant,
+    pin_all_cores_form_equals_single_thread,
 ]

@@ -1,6 +1,6 @@
 """gaf_cosdist_static: the entry point for callers that cannot allocate device
 memory (code inside a frozen memory pool, plug-ins called where cudaMalloc would
-stall the device).  It must give what gaf_cosdist gives, call after call, although
+stall the device).  It must give what gaf_cosdist and the CPU oracle give, call after call, although
 its scratch is one array shared by all calls that still holds the previous
 call's contents.  This file sorts last on purpose: a run that stops at the first
 failure has then already been through every other test."""
@@ -10,6 +10,7 @@ import pytest
 import torch
 
 import paper_2412_18052_b200 as gaf
+from oracle import gaf_oracle as orc
 from paper_2412_18052_b200 import workloads
 from parity import DIST_ATOL
 
@@ -42,6 +43,9 @@ def test_static_matches_workspace_entry_point_twice_in_a_row(dtype):
             gaf.gaf_cosdist_static(x, y, dist_s, stats_s)
             torch.cuda.synchronize()
             assert abs(float(dist_s.item()) - float(want_d.item())) <= DIST_ATOL
+            # ... and what the CPU oracle gives for the same bits
+            oracle_d, _ = orc.cosdist(workloads.as_numpy_bits(x), workloads.as_numpy_bits(y))
+            assert abs(float(dist_s.item()) - oracle_d) <= DIST_ATOL
             scale = float((want_s[1] * want_s[2]).sqrt().item()) + 1e-300
             assert float((stats_s - want_s).abs().max().item()) <= 1e-6 * scale
     # empty input and NULL stats
