@@ -602,7 +602,7 @@ def run_ours(args):
     cfg, steps = args.workload, args.steps
     peak, peak_kind = peak_bandwidth()
     m = measure_filter(torch, gaf, workloads, cfg, dev, args.tau, args.schedule, steps, args.warmup, nvml,
-                       rank=rank, D=args.D, barrier=barrier, want_warm=cfg in (1, 2))
+                       rank=rank, D=args.D, barrier=barrier, want_warm=cfg in (1, 2), want_c_loop=True)
     t = m["timing"]
     K, D, b, grad_bytes = m["K"], m["D"], m["b"], m["grad_bytes"]
     ms_per_step = max_over_ranks(t["ms_region"], dev) / steps
@@ -714,6 +714,7 @@ def run_ours(args):
             "ramp_calls": t["ramp_calls"],
             "e2e": e2e,
             "warm_l2": m.get("warm_l2"),
+            "c_loop": m.get("c_loop"),
             "gpu_launches": m["launches_per_step"] * steps,
             "clocks": t["clocks"],
             "cpu_baseline": cpu,

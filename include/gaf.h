@@ -73,7 +73,7 @@ enum {
                                    For K <= 8 the one-launch form is taken for binary32 inputs of
                                    at most 512 MB in all, and for bfloat16 inputs except 8
                                    gradients of more than 1 GB in all (tensor-core Gram then);
-                                   if the device refuses the co-resident launch, two launches. */
+                                   if the device refuses that launch, two launches. */
     GAF_SCHED_STEPWISE = 1,     /* streaming: one launch per step; each launch adds the
                                    gradient accepted at step t to the running sum and, in
                                    the same pass, takes the three dot products of the
@@ -84,13 +84,14 @@ enum {
                                    products are bilinear), then the accepted gradients are
                                    read once more to write g/c.  The distances agree with
                                    the stepwise schedule to rounding.  Two launches. */
-    GAF_SCHED_GRAM_FUSED = 3    /* Gram-first as ONE launch of a co-resident grid (K <= 8): the
-                                   same two passes, with the decisions exchanged through the
-                                   workspace between them, so that part of what the first pass
-                                   read (shared memory, L2) need not cross HBM again.  Identical
-                                   outputs to GAF_SCHED_GRAM.  GAF_ERR_UNSUPPORTED for K > 8 or on
-                                   a device without cooperative launches.  Its one internal wait
-                                   is bounded: GAF_STATUS_TIMEOUT if it ever runs out. */
+    GAF_SCHED_GRAM_FUSED = 3    /* Gram-first as ONE launch (K <= 8) of a grid sized to what the device
+                                   holds at once: the same two passes, every CTA taking the decisions
+                                   itself from the partial sums all CTAs left in the workspace, so that
+                                   part of what the first pass read (shared memory, L2) need not cross
+                                   HBM again.  Identical outputs to GAF_SCHED_GRAM.  GAF_ERR_UNSUPPORTED
+                                   for K > 8.  Its one wait on other CTAs is bounded:
+                                   GAF_STATUS_TIMEOUT if it ever runs out (it can only run out when
+                                   something else keeps part of the device busy for seconds). */
 };
 
 /* Bits of the device status word. */

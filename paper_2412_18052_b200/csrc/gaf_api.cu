@@ -38,7 +38,6 @@ struct DeviceInfo {
     int l2_bytes = 0;
     int smem_per_sm = 0;                // shared memory of one SM
     int smem_per_cta_max = 0;           // opt-in limit of one CTA
-    int cooperative = 0;                // cooperative launches supported
 };
 
 // What is worked out once per device and kept for the life of the process: the device's attributes and, per
@@ -73,8 +72,6 @@ bool device_info(DeviceInfo *out) {
         if (cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
             return GAF_ERR_CUDA;
         if (cudaDeviceGetAttribute(&d.smem_per_cta_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-            return GAF_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&d.cooperative, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess)
             return GAF_ERR_CUDA;
         return d.sms > 0 ? GAF_OK : GAF_ERR_CUDA;
     });
@@ -377,9 +374,18 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
     const int64_t per_elem = int64_t(KT) * int64_t(sizeof(T));
     const int64_t keep_elems = int64_t(di.l2_bytes) * kKeepL2Pct / 100 / per_elem;
     a.keep_from = a.D > keep_elems ? a.D - keep_elems : 0;
-    void *params[] = {&a};
-    const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kernel), dim3(int(grid)),
-                                                        dim3(kGsThreads), params, size_t(pl.dyn), st);
+    // The grid is no larger than what the device holds at once (occupancy above), so all its CTAs become
+    // resident and the one wait on other CTAs ends; it is bounded in any case.  Programmatic stream
+    // serialisation: the kernel waits for its predecessor on the stream itself (griddepcontrol.wait, first
+    // thing) and releases its successor once its decisions are taken.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned(grid)); cfg.blockDim = dim3(kGsThreads);
+    cfg.dynamicSmemBytes = size_t(pl.dyn); cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, a);
     if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     ++g_launches;
     return GAF_OK;
@@ -387,7 +393,6 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
 
 template <typename T>
 int launch_gram_fused(GramFusedArgs &a, int K, const DeviceInfo &di, cudaStream_t st) {
-    if (!di.cooperative) return GAF_ERR_UNSUPPORTED;
     switch (K) {
         case 2: return launch_gram_fused_kt<T, 2>(a, di, st);
         case 3: return launch_gram_fused_kt<T, 3>(a, di, st);
@@ -462,9 +467,8 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
 }
 
 // Whether the library's own choice is the one-launch form of the Gram-first schedule.
-bool auto_one_launch(int K, int64_t D, int dtype, const DeviceInfo &di) {
-    return di.cooperative && use_small_gram(K, D, dtype) &&
-           (dtype == GAF_BF16 || int64_t(K) * 4 * D <= kFusedMaxInputBytesF32);
+bool auto_one_launch(int K, int64_t D, int dtype) {
+    return use_small_gram(K, D, dtype) && (dtype == GAF_BF16 || int64_t(K) * 4 * D <= kFusedMaxInputBytesF32);
 }
 
 int check_workspace(const void *ws, size_t have, size_t need) {
@@ -630,7 +634,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
         // (the general CUDA-core Gram kernel beats the stepwise schedule up to 32 binary32 gradients)
         const bool fast_gram = K >= 2 && (K <= kGsMaxK || use_tensor_gram(K, D, dtype) ||
                                           (dtype == GAF_F32 && K <= kPanelAutoMaxK));
-        schedule = (fast_gram && ws_ok) ? (auto_one_launch(K, D, dtype, di) ? GAF_SCHED_GRAM_FUSED : GAF_SCHED_GRAM)
+        schedule = (fast_gram && ws_ok) ? (auto_one_launch(K, D, dtype) ? GAF_SCHED_GRAM_FUSED : GAF_SCHED_GRAM)
                                         : GAF_SCHED_STEPWISE;
     }
     if (K == 1) schedule = GAF_SCHED_STEPWISE;          // one gradient: it is the seed and the result
@@ -647,8 +651,8 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
         };
         int rc = run(schedule == GAF_SCHED_GRAM_FUSED);
         if (rc != GAF_OK && library_choice && schedule == GAF_SCHED_GRAM_FUSED) {
-            // the co-resident launch was refused (for example the device cannot hold the whole grid right
-            // now): the library's own choice falls back to the two-launch form, an explicit request does not
+            // the launch was refused (for example no CTA of this kernel fits an SM of this device): the
+            // library's own choice falls back to the two-launch form, an explicit request does not
             g_launches = 0;
             g_schedule = GAF_SCHED_GRAM;
             rc = run(false);
@@ -716,9 +720,9 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
             : launch_gram_first<__nv_bfloat16>(grads, K, D, dtype, tau, ord, macro_out, mask_out, dist_out,
                                                count_out, seed_out, base, di, one_launch, st);
     };
-    const bool one_launch = auto_one_launch(K, D, dtype, di);
+    const bool one_launch = auto_one_launch(K, D, dtype);
     int rc = run(one_launch);
-    if (rc != GAF_OK && one_launch) {       // co-resident launch refused: two launches
+    if (rc != GAF_OK && one_launch) {       // launch refused: two launches
         g_launches = 0;
         rc = run(false);
     }

@@ -28,9 +28,10 @@ struct Control {
     float stream_dist[GAF_MAX_K];       // streaming form: distance of arrival t
     uint8_t stream_mask[GAF_MAX_K];     // streaming form: decision of arrival t
     double norm_sq_sum;                 // stepwise and streaming forms: sum of |g_i|^2 over the accepted gradients
-    // One-launch Gram-first schedule: the word the waiting CTAs poll, alone in its cache line.
-    // Bits 16..31 call generation, 8..15 winning seed + 1 (0: no any-seed walk), 0..7 accept bits.
-    alignas(128) unsigned int fused_word;
+    // One-launch Gram-first schedule: the arrival counter its CTAs add to and poll, alone in its cache
+    // line.  Every call adds 4096 in all (one per CTA, the first CTA makes up the difference), so bits
+    // 12..31 count calls and bits 0..11 the CTAs of the running call that have arrived.
+    alignas(128) unsigned int fused_arrivals;
     unsigned int fused_pad[31];
 };
 constexpr size_t kControlBytes = 4096;  // sizeof(Control) rounded up

@@ -1,32 +1,42 @@
-// Gram-first schedule of Algorithm 1 as ONE persistent launch (K <= 8).
+// Gram-first schedule of Algorithm 1 as ONE launch (K <= 8).
 //
 // The two-launch form (gaf_gramfilter.cuh) reads every gradient once for the Gram
 // matrix and the accepted ones a second time for g/c (Eq. 5).  When the whole call
 // lasts tens of microseconds, what the second pass has to fetch again is a large part
-// of the cost.  Here one co-resident grid does both passes, so that part of what the
-// first pass read is still ON CHIP when the second pass starts:
+// of the cost.  Here one grid whose CTAs are all resident at once does both passes, so
+// that part of what the first pass read is still ON CHIP when the second pass starts:
 //   pass 1   every thread walks its vectors (grid-stride), accumulating the Gram
 //            partial sums exactly as gram_small_kernel does, and parks the raw loads
 //            of its FIRST R rounds in shared memory (the last rounds are the ones L2
 //            still holds afterwards: shared memory and L2 then keep different data);
-//   decide   per-CTA partials, last CTA to arrive totals them in fixed order, walks
-//            Algorithm 1 (Eq. 4 in binary64) on the Gram matrix and publishes the accept
-//            bits in one polled word; the other CTAs wait for it (bounded spin);
+//   decide   every CTA stores its partial sums and adds itself to an arrival counter;
+//            when the counter is full every CTA totals the partials in the same fixed
+//            order and walks Algorithm 1 (Eq. 4 in binary64) on the Gram matrix ITSELF --
+//            all CTAs get the same bits, nobody waits for a published result (one trip
+//            through L2 less than electing a CTA to decide); CTA 0 writes the outputs;
 //   pass 2   the same thread visits the same vectors: the rounds that were not parked
 //            from the last one down (the end of the vectors was loaded "keep in L2"),
 //            then the parked rounds straight from shared memory, adding the accepted
 //            gradients in processing order in binary32 and dividing by c.
 // Same sums, same order of additions as the two-launch form: identical outputs.
-// The grid must be co-resident (cooperative launch); every wait is bounded and ends in
-// GAF_STATUS_TIMEOUT.
+//
+// The grid is sized by the host to what the device holds at once.  The kernel is launched with
+// programmatic stream serialisation: it waits for whatever precedes it on the stream before it
+// touches memory, and lets the launch behind it be placed as soon as its own decisions are taken
+// (that launch waits in turn), which hides most of the launch latency of back-to-back calls.
+// The one wait on other CTAs is bounded and ends in GAF_STATUS_TIMEOUT.
 #pragma once
+
+#include <type_traits>
 
 #include "gaf_device.cuh"
 #include "gaf_gramfilter.cuh"
 
 namespace gaf {
 
-constexpr unsigned int kFusedSpinLimit = 1u << 23;   // polls of an L2 round trip plus a 40 ns sleep each: seconds
+constexpr unsigned int kFusedSpinLimit = 1u << 23;   // polls of an L2 round trip plus a 20 ns sleep each: seconds
+constexpr unsigned int kFusedCallUnit = 4096;        // what one call adds to the arrival counter in all
+constexpr int kFusedCallShift = 12;
 
 struct GramFusedArgs {
     const void *g[kGsMaxK];                 // processing order (original order in any-seed mode)
@@ -39,18 +49,24 @@ struct GramFusedArgs {
     ReplayArgs replay;                      // used when ring.K == 0
     RingArgs ring;                          // any-seed mode when ring.K > 0
     unsigned int spin_limit;                // polls a waiting CTA makes before it gives up
-    int test_withhold;                      // test hook, normally 0: the deciding CTA does not publish the
-                                            // decision word, so that every other CTA's wait runs out
+    int test_withhold;                      // test hook, normally 0: the waiting CTAs are never shown the full
+                                            // counter, so that every wait runs out
 };
 
-// The polled word carries its own payload, so no ordering with other memory is needed.
 __device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int *p) {
     unsigned int v;
     asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_relaxed_u32(unsigned int *p, unsigned int v) {
-    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Adds to a counter, ordered after everything this CTA wrote before (its threads' stores reach this
+// thread through the barrier in front of the call).
+__device__ __forceinline__ void red_release_add_u32(unsigned int *p, unsigned int v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 template <typename T> struct FusedVec;      // one 16-byte vector of a gradient, widened
@@ -80,6 +96,10 @@ __device__ __forceinline__ void store_vec_streaming(float *dst, const float (&v)
         __stcs(reinterpret_cast<float4 *>(dst) + h, make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]));
 }
 
+// Rounds of the second pass a thread keeps in flight, by the number of gradients it has to fetch per
+// round (8 loads of 16 bytes per thread at most, 2 rounds at least up to 4 gradients).
+template <int NN> struct FusedInFlight { static constexpr int U = NN <= 1 ? 8 : (NN == 2 ? 4 : (NN <= 4 ? 2 : 1)); };
+
 template <typename T, int KT>
 __global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1))
 gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
@@ -88,17 +108,21 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     extern __shared__ uint4 parked[];       // [round][gradient][thread]
     __shared__ double sacc[kGsThreads / 32][NP];
     __shared__ double sgram[KT * KT];
-    __shared__ bool is_last;
     __shared__ const T *list[kGsMaxK];      // accepted gradients in the order they are added
     __shared__ int list_row[kGsMaxK];       // ... and their row in `parked`
     __shared__ int n_list;                  // c, or -1 when the wait ran out
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     Control *ctl = a.replay.ctl;
 
-    // generation of the decision word before anybody can have published this call's
-    unsigned int gen0 = 0, decided = 0;
+    // Launched with programmatic stream serialisation, this grid may be placed while the launch before
+    // it on the stream is still winding down: nothing that launch (or the producer of the gradients)
+    // wrote may be touched before it has completed.  A no-op after an ordinary predecessor.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // call generation before this CTA has arrived: it cannot change until every CTA has, this one included
+    unsigned int gen0 = 0;
     if (tid == 0) {
-        gen0 = ld_relaxed_u32(&ctl->fused_word) >> 16;
+        gen0 = ld_relaxed_u32(&ctl->fused_arrivals) >> kFusedCallShift;
         if (blockIdx.x == 0) ctl->status = 0;
     }
     for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
@@ -188,94 +212,95 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
         a.partials[(size_t)tid * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     }
     __syncthreads();
+
+    // ---- decide: arrive, wait until every CTA has, then total the partials and walk Algorithm 1 here ----
     if (tid == 0) {
-        is_last = take_last_ticket(&ctl->ticket, gridDim.x);
+        red_release_add_u32(&ctl->fused_arrivals, blockIdx.x == 0 ? kFusedCallUnit - (gridDim.x - 1) : 1u);
+        unsigned int polls = 0;
+        bool ok = true;
+        // (the acquire orders the loads of the partials below, through the barrier, after every CTA's stores)
+        while ((ld_acquire_u32(&ctl->fused_arrivals) >> kFusedCallShift) == gen0 || a.test_withhold) {
+            __nanosleep(20);
+            if (++polls > a.spin_limit) { ok = false; break; }
+        }
+        n_list = ok ? 0 : -1;
+        if (!ok) atomicOr(&ctl->status, GAF_STATUS_TIMEOUT);
     }
     __syncthreads();
-
-    // ---- decide: last CTA totals the partials in fixed order and walks Algorithm 1 ----
-    if (is_last) {
-        total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
-        __syncthreads();
-        // the accept bits go out first, in the polled word itself; the outputs follow
-        auto notice = [&](int seed, unsigned long long bits) {
-            const unsigned int word = ((gen0 + 1u) << 16) | ((unsigned int)(seed + 1) << 8) | (unsigned int)(bits & 0xFFull);
-            decided = word;
-            if (!a.test_withhold) st_relaxed_u32(&ctl->fused_word, word);
-        };
-        if (a.ring.K > 0) {
-            __shared__ RingTable<KT> ring_table;
-            ring_replay_parallel<KT>(a.ring, sgram, ring_table, notice);
-        } else {
-            __shared__ ReplayTable table;
-            replay_on_gram_parallel<KT>(a.replay, sgram, table, [&](unsigned long long bits) { notice(-1, bits); });
-        }
-    }
-    if (tid == 0) {
-        unsigned int word = decided;
-        bool ok = true;
-        if (!is_last) {
-            unsigned int polls = 0;
-            while (((word = ld_relaxed_u32(&ctl->fused_word)) >> 16) == gen0) {
-                __nanosleep(40);
-                if (++polls > a.spin_limit) { ok = false; break; }
-            }
-        }
-        if (!ok) {
-            atomicOr(&ctl->status, GAF_STATUS_TIMEOUT);
-            n_list = -1;
-        } else {
-            const unsigned int bits = word & 0xFFu;
-            const int seed = (int)((word >> 8) & 0xFFu) - 1;
+    if (n_list < 0) return;                 // every CTA has arrived all the same: the counter is whole again
+    const bool publisher = blockIdx.x == 0;
+    total_gram_partials<KT>(a.partials, gridDim.x, sgram, publisher ? a.gram : nullptr);
+    __syncthreads();
+    {
+        // every CTA takes the same sums in the same order, hence the same decisions; one of them writes them out
+        auto take = [&](int seed, unsigned long long bits) {
             const int start = seed < 0 ? 0 : seed;
             int n = 0;
             for (int t = 0; t < KT; ++t) {
                 const int i = (start + t) % KT;
-                if ((bits >> i) & 1u) { list[n] = static_cast<const T *>(a.g[i]); list_row[n] = i; ++n; }
+                if ((bits >> i) & 1ull) { list[n] = static_cast<const T *>(a.g[i]); list_row[n] = i; ++n; }
             }
             n_list = n;
+        };
+        if (a.ring.K > 0) {
+            __shared__ RingTable<KT> ring_table;
+            ring_replay_parallel<KT>(a.ring, sgram, ring_table, take, publisher);
+        } else {
+            __shared__ ReplayTable table;
+            replay_on_gram_parallel<KT>(a.replay, sgram, table, [&](unsigned long long bits) { take(-1, bits); }, publisher);
         }
     }
     __syncthreads();
     const int n = n_list;
-    if (n < 0) return;
     const float cdiv = (float)n;
+    // the launch behind this one on the stream may be placed from here on (it waits for this grid itself)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    // ---- pass 2a: the rounds that were not parked, last first (what pass 1 read last is what
-    //      L2 still holds), two rounds in flight per thread ----
-    constexpr int U = 2;
-    for (int64_t j0 = rounds - 1; j0 >= parked_rounds; j0 -= U) {
-        int64_t ju[U];
+    // ---- pass 2a: the rounds that were not parked, last first (what pass 1 read last is what L2 still
+    //      holds), several rounds in flight per thread; specialised on the number of accepted gradients ----
+    auto pass2a = [&](auto nn_tag) {
+        constexpr int NN = decltype(nn_tag)::value;
+        constexpr int U = FusedInFlight<NN>::U;
+        for (int64_t j0 = rounds - 1; j0 >= parked_rounds; j0 -= U) {
+            int64_t q[U];
+            bool ok[U];
+            uint4 w[U][NN];
 #pragma unroll
-        for (int u = 0; u < U; ++u) ju[u] = j0 - u >= parked_rounds ? j0 - u : -1;
-        int64_t q[U];
-        bool ok[U];
-        uint4 w[U][KT];
+            for (int u = 0; u < U; ++u) {
+                const int64_t ju = j0 - u;
+                q[u] = warp_first + ju * stride + lane;
+                ok[u] = ju >= parked_rounds && q[u] < n_vec;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            q[u] = warp_first + ju[u] * stride + lane;
-            ok[u] = ju[u] >= 0 && q[u] < n_vec;
+                for (int i = 0; i < NN; ++i)
+                    if (ok[u]) w[u][i] = ld16_policy(list[i] + q[u] * N, pol_first);
+            }
 #pragma unroll
-            for (int i = 0; i < KT; ++i)
-                if (ok[u] && i < n) w[u][i] = ld16_policy(list[i] + q[u] * N, pol_first);
-        }
+            for (int u = 0; u < U; ++u)
+                if (ok[u]) {
+                    float v[N];
+                    FusedVec<T>::widen(w[u][0], v);
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (ok[u]) {
-                float v[N];
-                FusedVec<T>::widen(w[u][0], v);
-#pragma unroll
-                for (int i = 1; i < KT; ++i)
-                    if (i < n) {
+                    for (int i = 1; i < NN; ++i) {
                         float x[N];
                         FusedVec<T>::widen(w[u][i], x);
 #pragma unroll
                         for (int k = 0; k < N; ++k) v[k] += x[k];
                     }
 #pragma unroll
-                for (int k = 0; k < N; ++k) v[k] = v[k] / cdiv;
-                store_vec_streaming<N>(a.out + q[u] * N, v);
-            }
+                    for (int k = 0; k < N; ++k) v[k] = v[k] / cdiv;
+                    store_vec_streaming<N>(a.out + q[u] * N, v);
+                }
+        }
+    };
+    switch (n) {
+        case 1: pass2a(std::integral_constant<int, 1>()); break;
+        case 2: if constexpr (KT >= 2) pass2a(std::integral_constant<int, 2>()); break;
+        case 3: if constexpr (KT >= 3) pass2a(std::integral_constant<int, 3>()); break;
+        case 4: if constexpr (KT >= 4) pass2a(std::integral_constant<int, 4>()); break;
+        case 5: if constexpr (KT >= 5) pass2a(std::integral_constant<int, 5>()); break;
+        case 6: if constexpr (KT >= 6) pass2a(std::integral_constant<int, 6>()); break;
+        case 7: if constexpr (KT >= 7) pass2a(std::integral_constant<int, 7>()); break;
+        default: if constexpr (KT >= 8) pass2a(std::integral_constant<int, 8>()); break;
     }
     // ---- pass 2b: the parked rounds, from shared memory ----
     for (int64_t j = 0; j < parked_rounds; ++j) {

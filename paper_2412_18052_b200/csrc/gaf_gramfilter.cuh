@@ -90,7 +90,8 @@ __device__ __forceinline__ unsigned long long replay_on_gram(const ReplayArgs &r
 // and thread 0 then only follows the decisions through the table.  Every case repeats the sums of
 // the sequential walk in the same order, so the results are the same to the last bit.
 // All threads of the block call (blockDim.x >= 128).  `early(bits)` is called by thread 0 as soon as
-// the accept bits are known, before the outputs are written.
+// the accept bits are known, before the outputs are written.  With `publish` false nothing is written
+// to global memory (the one-launch schedule runs the walk in every CTA and lets one of them publish).
 struct ReplayTable {
     double d[127], p[127], na[127];
     unsigned char accept[127], status[127];
@@ -100,7 +101,7 @@ struct NoEarlyBits {
 };
 template <int KT, typename Early = NoEarlyBits>
 __device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, const double *gram, ReplayTable &tb,
-                                                        Early early = Early()) {
+                                                        Early early = Early(), bool publish = true) {
     constexpr int K = KT;
     const int tid = threadIdx.x;
     constexpr int cases = (1 << (K - 1)) - 1;
@@ -147,6 +148,7 @@ __device__ __forceinline__ void replay_on_gram_parallel(const ReplayArgs &r, con
         }
         const unsigned long long bits = 1ull | ((unsigned long long)m << 1);
         early(bits);
+        if (!publish) return;
         Control *c = r.ctl;
         int status = 0, count = 1;
         c->decision[0] = 1;
@@ -258,7 +260,8 @@ __device__ __forceinline__ void ring_replay_on_gram(const RingArgs &r, const vol
 // ORIGINAL index (step v of seed s is gradient (s + v) mod K), one thread per seed then follows its
 // decisions through the table, and thread 0 picks the largest count (ties to the smallest seed) and
 // publishes.  Same sums in the same order as ring_walk_one_seed: identical outputs.
-// All threads of the block call; `early(seed, bits)` as in ring_replay_on_gram.
+// All threads of the block call; `early(seed, bits)` as in ring_replay_on_gram; `publish` as in
+// replay_on_gram_parallel.
 template <int KT>
 struct RingTable {
     static constexpr int kCases = (1 << (KT - 1)) - 1;          // per seed
@@ -269,7 +272,7 @@ struct RingTable {
 };
 template <int KT, typename Early = NoEarlyNotice>
 __device__ __forceinline__ void ring_replay_parallel(const RingArgs &r, const double *gram, RingTable<KT> &tb,
-                                                     Early early = Early()) {
+                                                     Early early = Early(), bool publish = true) {
     constexpr int K = KT, C = RingTable<KT>::kCases;
     for (int idx = threadIdx.x; idx < K * C; idx += blockDim.x) {
         const int s = idx / C, cs = idx - s * C;
@@ -324,6 +327,7 @@ __device__ __forceinline__ void ring_replay_parallel(const RingArgs &r, const do
         for (int t = 1; t < K; ++t)
             if ((steps >> (t - 1)) & 1u) bits |= 1ull << ((best + t) % K);
         early(best, bits);
+        if (!publish) return;
         int status = 0;
         unsigned int m = 0;
         if (r.dist_out) r.dist_out[best] = 0.0f;

@@ -339,7 +339,7 @@ def test_bounded_waits_run_out_and_the_workspace_recovers(ws):
     so every wait runs out.  The call must end by itself with GAF_STATUS_TIMEOUT, and the next
     ordinary call on the same workspace must be correct."""
     cases = [
-        # one-launch Gram-first schedule: the deciding CTA does not publish the decision word
+        # one-launch Gram-first schedule: the waiting CTAs are never shown the full arrival counter
         (_mix(4, 600_011, "f32", seed=11, rho=[0.8, 0.6, -0.2, 0.7]), gaf.GAF_SCHED_GRAM_FUSED),
         (_mix(8, 300_007, "bf16", seed=12), gaf.GAF_SCHED_GRAM_FUSED),
         # tensor-core Gram pipeline: the first tile's barrier never completes
