@@ -6,11 +6,13 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "../../include/gaf.h"
 #include "gaf_bucketed.cuh"
 #include "gaf_device.cuh"
 #include "gaf_fused.cuh"
+#include "gaf_gram_mma.cuh"
 #include "gaf_gram_panel.cuh"
 #include "gaf_gram_tc.cuh"
 #include "gaf_gramfilter.cuh"
@@ -142,15 +144,13 @@ int stream_grid(int64_t D, int threads, int sms) {
     return int(need < cap ? need : cap);
 }
 
-// Which Gram kernel.  The tensor-core kernel pays off from 8 bfloat16 gradients on: with fewer, most
-// of each 128-row MMA tile is padding and the register-tiled kernel is faster at every length
-// (measured: 4 gradients of 5e8 elements, 1.85 ms against 1.41 ms).  With exactly 8 it wins only
-// once the vectors are long enough for the one-launch schedule to have lost its edge.
-constexpr int64_t kTcMinBytesK8 = int64_t(1) << 30;
+// Which Gram kernel.  The 128-row tcgen05 tile pays off from 9 bfloat16 gradients on.  Up to 8 the one-pass
+// kernels for few gradients are faster at every length: with exactly 8, where the 128 x 128 product keeps 1/16 of
+// its work, the warp-level MMA kernel streams 16 GB of inputs at 6.6 TB/s against 5.2 TB/s (measured).
 constexpr int kPanelAutoMaxK = 32;
 bool use_tensor_gram(int K, int64_t D, int dtype) {
-    if (dtype != GAF_BF16 || K < kGsMaxK || K > kTcMaxK) return false;
-    return K > kGsMaxK || int64_t(K) * 2 * D > kTcMinBytesK8;
+    (void)D;
+    return dtype == GAF_BF16 && K > kGsMaxK && K <= kTcMaxK;
 }
 bool use_small_gram(int K, int64_t D, int dtype) {
     return K >= 2 && K <= kGsMaxK && !use_tensor_gram(K, D, dtype);
@@ -277,12 +277,17 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
 }
 
 template <typename T, int KT>
-int launch_gram_small_kt(const GramSmallArgs &a, const DeviceInfo &di, cudaStream_t st) {
+int launch_gram_small_kt(GramSmallArgs a, const DeviceInfo &di, cudaStream_t st) {
+    // 7 or 8 bfloat16 gradients go through the warp-level tensor-core kernel (with fewer, the lanes of the
+    // absent rows fetch nothing and too few bytes are in flight: measured slower than the register tile)
+    constexpr bool kMma = std::is_same<T, __nv_bfloat16>::value && KT >= 7;
+    void (*kernel)(GramSmallArgs) = nullptr;
+    if constexpr (kMma) kernel = gram_mma_kernel<KT>;
+    else kernel = gram_small_kernel<T, KT>;
     static PerDevice<OccPlan> table;
-    plan_once(table.plan[di.dev], table.ready[di.dev], [](OccPlan &pl) {
+    plan_once(table.plan[di.dev], table.ready[di.dev], [kernel](OccPlan &pl) {
         int occ = 1;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, gram_small_kernel<T, KT>, kGsThreads, 0) !=
-            cudaSuccess || occ < 1)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kGsThreads, 0) != cudaSuccess || occ < 1)
             occ = 1;
         pl.occ = occ > 2 ? 2 : occ;
         return GAF_OK;
@@ -290,10 +295,15 @@ int launch_gram_small_kt(const GramSmallArgs &a, const DeviceInfo &di, cudaStrea
     const int occ = table.plan[di.dev].occ;
     int64_t grid = int64_t(di.sms) * occ;
     if (grid > kGsMaxCtas) grid = kGsMaxCtas;
-    const int64_t work = (a.D / GsVec<T>::N + kGsThreads - 1) / kGsThreads;
+    // elements one CTA consumes per trip of its loop
+    const int64_t per_cta = kMma ? int64_t(kGsThreads / 32) * kMmaTileElems * 2 : int64_t(kGsThreads) * GsVec<T>::N;
+    const int64_t work = (a.D + per_cta - 1) / per_cta;
     if (grid > work) grid = work;
     if (grid < 1) grid = 1;
-    gram_small_kernel<T, KT><<<int(grid), kGsThreads, 0, st>>>(a);
+    // long vectors: runs of several trips per CTA (address-translation locality), once every CTA gets
+    // at least eight such runs; otherwise one trip at a time
+    a.mma_run = (kMma && a.D >= int64_t(8) * kMmaLongRun / 2 * per_cta * grid) ? kMmaLongRun : 2;
+    kernel<<<int(grid), kGsThreads, 0, st>>>(a);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }
@@ -322,8 +332,10 @@ constexpr int kKeepL2Pct = 10;          // share of L2 the Gram pass asks to kee
 constexpr int kParkBytesPerSm = 128 << 10;
 // AUTO takes the one-launch form for binary32 inputs up to this many bytes in all: beyond, what stays
 // on chip between the passes is a negligible share and the two-launch form is as fast or slightly
-// faster.  For bfloat16 the one-launch form stays ahead at every length measured.
+// faster.  For bfloat16 with up to 6 gradients the one-launch form stays ahead at every length measured;
+// with 7 or 8 the two-launch form on the warp-level MMA Gram kernel overtakes it near 1 GB of inputs.
 constexpr int64_t kFusedMaxInputBytesF32 = int64_t(512) << 20;
+constexpr int64_t kFusedMaxInputBytesBf16Mma = int64_t(1) << 30;
 
 template <typename T, int KT>
 int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st) {
@@ -459,6 +471,12 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
     for (int t = 0; t < K; ++t) m.g[t] = g[ord[t]];
     m.K = K; m.D = D; m.out = macro_out; m.ctl = ctl;
     const int grid = stream_grid(D, kMsThreads, sms);
+    {
+        // runs of 8 chunks per CTA once every CTA gets at least eight such runs, else one trip at a time
+        const int per_trip = sizeof(T) == 2 ? 2 : 1;
+        const int64_t chunks = (D / kOct + kMsThreads - 1) / kMsThreads;
+        m.run = chunks >= int64_t(8) * kMsLongRun * grid ? kMsLongRun : per_trip;
+    }
     // the blocks may be placed while the Gram pass winds down (its last CTA is still totalling partials)
     const cudaError_t err = launch_dependent(masked_mean_kernel<T>, grid, kMsThreads, st, m);
     ++g_launches;
@@ -468,7 +486,9 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
 
 // Whether the library's own choice is the one-launch form of the Gram-first schedule.
 bool auto_one_launch(int K, int64_t D, int dtype) {
-    return use_small_gram(K, D, dtype) && (dtype == GAF_BF16 || int64_t(K) * 4 * D <= kFusedMaxInputBytesF32);
+    if (!use_small_gram(K, D, dtype)) return false;
+    if (dtype == GAF_F32) return int64_t(K) * 4 * D <= kFusedMaxInputBytesF32;
+    return K < 7 || int64_t(K) * 2 * D <= kFusedMaxInputBytesBf16Mma;
 }
 
 int check_workspace(const void *ws, size_t have, size_t need) {

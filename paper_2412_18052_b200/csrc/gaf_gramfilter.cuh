@@ -24,6 +24,7 @@ constexpr int kGsMaxCtas = 296;
 constexpr int kGsPartialStride = 320;       // per-CTA partials are stored [pair][CTA]: the totalling loads coalesce
 constexpr int kGsFlushEvery = 16;           // iterations between binary64 flushes
 constexpr int kMsThreads = 512;
+constexpr int kMsLongRun = 8;                // chunks per run of the masked-mean pass on long vectors
 constexpr int kReplayMaxK = 8;               // the table form of the walk: 2^(K-1) - 1 cases
 
 struct ReplayArgs {
@@ -361,6 +362,7 @@ struct GramSmallArgs {
     float *pair_dist_out;                   // pairwise mode: K x K distances instead of the walk
     double *pair_gram_out;                  // pairwise mode: optional copy of the Gram matrix
     RingArgs ring;                          // any-seed mode when ring.K > 0 (rows are in original order)
+    int mma_run;                            // gram_mma_kernel: trips per run of a CTA (even, >= 2)
 };
 
 // 16-byte read-only load with an explicit L2 eviction policy.
@@ -467,12 +469,67 @@ template <> struct GsAcc<float, 4> { using type = double; static constexpr bool 
 __device__ __forceinline__ float gs_fma(float a, float b, float s) { return fmaf(a, b, s); }
 __device__ __forceinline__ double gs_fma(float a, float b, double s) { return fma((double)a, (double)b, s); }
 
+// What every one-pass Gram kernel for K <= 8 does once its warps have left their sums in
+// sacc[warp][pair] (upper triangle, row-major pair index): per-CTA partial sums in a fixed order,
+// last-CTA election, fixed-order totals, then the walk of Algorithm 1 (or the any-seed walks, or the
+// pairwise distances).  All threads of the block call.
+template <int KT>
+__device__ __forceinline__ void gram_small_tail(const GramSmallArgs &a, double (*sacc)[KT * (KT + 1) / 2]) {
+    constexpr int NP = KT * (KT + 1) / 2;
+    __shared__ bool is_last;
+    // the streaming part of this CTA is over: a kernel launched as a programmatic dependent
+    // (the masked-mean pass) may start occupying SMs; it still waits for this whole grid
+    // before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x < NP) {
+        // the 16 warps' sums in four short chains (a fixed order, so still reproducible)
+        double s4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            s4[c] = sacc[4 * c][threadIdx.x];
+#pragma unroll
+            for (int w = 1; w < 4; ++w) s4[c] += sacc[4 * c + w][threadIdx.x];
+        }
+        a.partials[(size_t)threadIdx.x * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = take_last_ticket(&a.replay.ctl->ticket, gridDim.x);
+    __syncthreads();
+    if (!is_last) return;
+
+    // last CTA: fixed-order totals (one warp per pair; all of a lane's loads are issued together,
+    // this is the serial tail of the call), then the scalar walk out of shared memory
+    __shared__ double sgram[KT * KT];
+    total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
+    __syncthreads();
+    if (a.ring.K > 0) {
+        __shared__ RingTable<KT> ring_table;
+        ring_replay_parallel<KT>(a.ring, sgram, ring_table);
+        return;
+    }
+    if (a.pair_dist_out == nullptr) {
+        __shared__ ReplayTable table;
+        replay_on_gram_parallel<KT>(a.replay, sgram, table);
+        return;
+    }
+    // pairwise mode: Eq. 4 for every pair
+    if (threadIdx.x < KT * KT) {
+        const int i = threadIdx.x / KT, j = threadIdx.x % KT;
+        const double gii = sgram[i * KT + i], gjj = sgram[j * KT + j], gij = sgram[threadIdx.x];
+        int status = 0;
+        const double d = (i == j && gii > 0.0) ? 0.0 : cosine_distance(gij, gii, gjj, &status);
+        a.pair_dist_out[threadIdx.x] = (float)d;
+        if (a.pair_gram_out) a.pair_gram_out[threadIdx.x] = gij;
+        if (status) atomicOr(&a.replay.ctl->status, status);
+    }
+}
+
 template <typename T, int KT>
 __global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1)) gram_small_kernel(const __grid_constant__ GramSmallArgs a) {
     constexpr int NP = KT * (KT + 1) / 2;   // upper triangle
     constexpr int N = GsVec<T>::N;
     __shared__ double sacc[kGsThreads / 32][NP];
-    __shared__ bool is_last;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (blockIdx.x == 0 && threadIdx.x == 0) a.replay.ctl->status = 0;      // first kernel of the operation
     for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
@@ -542,52 +599,7 @@ __global__ void __launch_bounds__(kGsThreads, (KT <= 4 ? 2 : 1)) gram_small_kern
             for (int c = r; c < KT; ++c, ++p) acc[p] = gs_fma(x[r], x[c], acc[p]);
     }
     flush();
-    // the streaming part of this CTA is over: a kernel launched as a programmatic dependent
-    // (the masked-mean pass) may start occupying SMs; it still waits for this whole grid
-    // before it reads anything
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    __syncthreads();
-    if (threadIdx.x < NP) {
-        // the 16 warps' sums in four short chains (a fixed order, so still reproducible)
-        double s4[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            s4[c] = sacc[4 * c][threadIdx.x];
-#pragma unroll
-            for (int w = 1; w < 4; ++w) s4[c] += sacc[4 * c + w][threadIdx.x];
-        }
-        a.partials[(size_t)threadIdx.x * kGsPartialStride + blockIdx.x] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) is_last = take_last_ticket(&a.replay.ctl->ticket, gridDim.x);
-    __syncthreads();
-    if (!is_last) return;
-
-    // last CTA: fixed-order totals (one warp per pair; all of a lane's loads are issued together,
-    // this is the serial tail of the call), then the scalar walk out of shared memory
-    __shared__ double sgram[KT * KT];
-    total_gram_partials<KT>(a.partials, gridDim.x, sgram, a.gram);
-    __syncthreads();
-    if (a.ring.K > 0) {
-        __shared__ RingTable<KT> ring_table;
-        ring_replay_parallel<KT>(a.ring, sgram, ring_table);
-        return;
-    }
-    if (a.pair_dist_out == nullptr) {
-        __shared__ ReplayTable table;
-        replay_on_gram_parallel<KT>(a.replay, sgram, table);
-        return;
-    }
-    // pairwise mode: Eq. 4 for every pair
-    if (threadIdx.x < KT * KT) {
-        const int i = threadIdx.x / KT, j = threadIdx.x % KT;
-        const double gii = sgram[i * KT + i], gjj = sgram[j * KT + j], gij = sgram[threadIdx.x];
-        int status = 0;
-        const double d = (i == j && gii > 0.0) ? 0.0 : cosine_distance(gij, gii, gjj, &status);
-        a.pair_dist_out[threadIdx.x] = (float)d;
-        if (a.pair_gram_out) a.pair_gram_out[threadIdx.x] = gij;
-        if (status) atomicOr(&a.replay.ctl->status, status);
-    }
+    gram_small_tail<KT>(a, sacc);
 }
 
 // Scalar walk as its own launch (Gram matrix produced by the tiled pairwise kernels).
@@ -647,12 +659,18 @@ struct MaskedMeanArgs {
     int64_t D;
     float *out;
     const Control *ctl;
+    int run;                                // chunks (of one CTA's 512 groups of 8 elements) a CTA takes in a row
 };
 
 // out = (((g_0 + g_a) + g_b) + ...) / c over the accepted steps a < b < ..., binary32,
 // in processing order: the same association as the streaming schedule.  The vector is
 // walked from its END: the Gram pass that ran just before walked it from the start, so
-// its last-read lines are the ones still in L2.
+// its last-read lines are the ones still in L2.  A CTA takes `run` consecutive chunks, then
+// jumps ahead by the whole grid's share: with run = U the grid works on one compact window of
+// every vector at any moment (short vectors: every CTA has work); on long vectors longer runs
+// keep an SM inside the same pages for several trips, which the address translation needs
+// (12 GB through this pass: 5.5 TB/s with run = U, measured, against the 6.5 TB/s it reaches
+// on shorter vectors).
 template <typename T>
 __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid_constant__ MaskedMeanArgs a) {
     __shared__ const T *list[GAF_MAX_K];
@@ -681,19 +699,21 @@ __global__ void __launch_bounds__(kMsThreads, 2) masked_mean_kernel(const __grid
     const int n = n_list;
     const float cdiv = cdiv_s;
     const int64_t n_oct = a.D / kOct;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     // U groups of 8 elements per thread and round (two for 2-byte inputs, so that as many bytes
     // are in flight as with 4-byte inputs); loads stay packed until they are added
     constexpr int U = sizeof(T) == 2 ? 2 : 1;
     constexpr int kChunk = 3;                       // further gradients fetched together
-    for (int64_t o0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o0 < n_oct; o0 += stride * U) {
+    const int64_t n_chunks = (n_oct + kMsThreads - 1) / kMsThreads;
+    const int64_t run = a.run;
+    for (int64_t base = (int64_t)blockIdx.x * run; base < n_chunks; base += (int64_t)gridDim.x * run)
+    for (int64_t rr = 0; rr < run && base + rr < n_chunks; rr += U) {
         int64_t e[U];
         bool ok[U];
         RawOct<T> first[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int64_t o = o0 + u * stride;
-            ok[u] = o < n_oct;
+            const int64_t o = (base + rr + u) * kMsThreads + threadIdx.x;
+            ok[u] = rr + u < run && o < n_oct;
             e[u] = (n_oct - 1 - (ok[u] ? o : 0)) * kOct;
             if (ok[u]) first[u] = RawOct<T>::load(list[0], e[u]);
         }

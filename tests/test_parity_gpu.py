@@ -538,6 +538,21 @@ def test_auto_schedule_choice(ws):
         g[i::8] = 1.0
     gaf.gaf_filter_accumulate(big, 0.97, ws)
     assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM
+    # 8 bfloat16 gradients of more than 1 GB in all: two launches as well (warp-level MMA Gram kernel, masked mean)
+    big = [torch.zeros(70_000_000, device="cuda", dtype=torch.bfloat16) for _ in range(8)]
+    for i, g in enumerate(big):
+        g[i::8] = 1.0
+    gaf.gaf_filter_accumulate(big, 0.97, ws)
+    assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM and gaf.gaf_last_launch_count() == 2
+
+
+def test_mma_gram_kernel_long_runs(ws):
+    """7 and 8 bfloat16 gradients take the warp-level tensor-core Gram kernel; from about 19 M elements on its
+    CTAs walk the vectors in runs of several trips.  Both mappings, with ragged ends, against the oracle."""
+    for K, D in ((8, 20_000_000 + 37), (7, 19_500_003), (8, 2_500_000 + 63), (7, 64 * 16 * 296 * 2 + 5)):
+        w = _mix(K, D, "bf16", seed=600 + K)
+        check_filter(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM)
+        check_pairwise(w.grads, ws)
 
 
 def test_gram_sums_of_few_fp32_gradients_are_exact_to_binary64_rounding(ws):
