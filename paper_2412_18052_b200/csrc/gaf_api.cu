@@ -191,7 +191,25 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
                                                       2 * gram_matrix_bytes(K));
     a.gram_out = gram_out;
     a.ctl = reinterpret_cast<Control *>(base);
-    if (use_tensor_gram(K, D, dtype)) {
+    if (use_tensor_gram(K, D, dtype) && K <= kWideMaxK) {
+        // 9..16 bfloat16 gradients: warp-level MMAs fed straight from the global loads, two CTAs per SM
+        GramWideArgs w{};
+        for (int i = 0; i < K; ++i) w.g[i] = grads[i];
+        w.K = K; w.D = D; w.keep_from = D; w.partials = a.partials; w.ctl = a.ctl;
+        const int64_t per_cta = int64_t(kWideThreads / 32) * kMmaTileElems;      // elements per trip of one CTA
+        int64_t grid = int64_t(sms) * 2;
+        if (grid > kGramMaxSlices) grid = kGramMaxSlices;
+        const int64_t work = (D + per_cta - 1) / per_cta;
+        if (grid > work) grid = work;
+        if (grid < 1) grid = 1;
+        a.slices = int(grid);
+        // runs of 8 trips per CTA on long vectors (address-translation locality), one trip at a time otherwise
+        w.run = D >= int64_t(32) * kMmaLongRun * per_cta * grid ? kMmaLongRun : 1;
+        void (*kernel)(GramWideArgs) = gram_mma_wide_kernel;
+        const int dyn = (kWideThreads / 32) * 2 * 128 * int(sizeof(double));       // [warp][tile][lane][4] doubles: 32 KB
+        kernel<<<int(grid), kWideThreads, dyn, st>>>(w);
+        ++g_launches;
+    } else if (use_tensor_gram(K, D, dtype)) {
         // tensor cores: one CTA per SM, each with a contiguous slice of D
         GramTcArgs t{};
         for (int i = 0; i < K; ++i) t.g[i] = grads[i];

@@ -126,4 +126,144 @@ __global__ void __launch_bounds__(kMmaThreads, 2) gram_mma_kernel(const __grid_c
     gram_small_tail<KT>(a, sacc);
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same idea for 9..16 bfloat16 gradients: two blocks of 8 rows.  Lane (g, t) loads 8 elements of
+// gradient g and of gradient g + 8 -- two loads of 16 bytes per 32-element chunk -- and those registers
+// are at once the A fragment of the 16-row block (rows g and g + 8) and the B fragments of the two
+// 8-column blocks.  Two 16 x 8 tiles cover the upper triangle: 4 MMAs per 32 elements, three quarters of
+// whose work is kept, against one eighth for the 128 x 128 tcgen05 tile with 16 gradients.  No
+// shared-memory staging, no barriers in the streaming loop.  Measured at D = 11.2 M: 54 / 58 / 64 us with
+// 9 / 12 / 16 gradients against 64 / 69 / 74 us on the tcgen05 kernel.  The form with 3 and 4 row blocks
+// (up to 32 gradients, 12 MMAs per 32 elements) was built and measured as well: 210 us against 145 us at 32
+// gradients -- the warp-level MMA rate of this GPU (about 150 TFLOP/s here) is what 32 gradients need at
+// HBM speed, so from 17 gradients on the tcgen05 tile stays.
+// Per-CTA partial sums go out in the [tile pair][slice][64] layout of the tiled Gram kernels
+// (gaf_pairwise.cuh), so gram_finish_kernel totals them.
+
+struct GramWideArgs {
+    const void *g[16];
+    int K;
+    int64_t D;
+    int64_t keep_from;
+    double *partials;           // [tile pair][slice][64]
+    Control *ctl;
+    int run;                    // tiles per warp a CTA takes in a row (even)
+};
+
+constexpr int kWideThreads = 512;
+constexpr int kWideMaxK = 16;
+
+__device__ __forceinline__ void mma_bf16_16816_full(float (&c)[4], unsigned int a0, unsigned int a1, unsigned int a2,
+                                                    unsigned int a3, unsigned int b0, unsigned int b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(kWideThreads, 2) gram_mma_wide_kernel(const __grid_constant__ GramWideArgs a) {
+    constexpr int NB = 2;                           // blocks of 8 rows
+    constexpr int NT = 2;                           // 16 x 8 tiles: columns 0..7 and 8..15
+    extern __shared__ double wide_red[];            // [warp][tile][lane][4] at the end
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.ctl->status = 0;            // first kernel of the operation
+
+    const unsigned short *rowp[NB];
+    bool have[NB];
+#pragma unroll
+    for (int m = 0; m < NB; ++m) {
+        have[m] = g + 8 * m < a.K;
+        rowp[m] = static_cast<const unsigned short *>(a.g[have[m] ? g + 8 * m : 0]);
+    }
+    const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
+    const int64_t n_tiles = a.D / kMmaTileElems;
+    float c[NT][4];
+    double d[NT][4];
+#pragma unroll
+    for (int i = 0; i < NT; ++i)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { c[i][k] = 0.f; d[i][k] = 0.0; }
+    int chain = 0;
+    constexpr int kWarps = kWideThreads / 32;
+    const int run = a.run;
+    const int64_t cta_run_tiles = (int64_t)run * kWarps, grid_run_tiles = cta_run_tiles * gridDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * cta_run_tiles; base < n_tiles; base += grid_run_tiles) {
+        for (int rr = 0; rr < run; ++rr) {
+            const int64_t tile = base + (int64_t)rr * kWarps + warp;
+            if (tile >= n_tiles) break;
+            // one tile of 64 elements: two chunks of 32, all 2 NB loads issued before the first MMA
+            const int64_t e0 = tile * kMmaTileElems + t * 8;
+            const uint64_t pol = (e0 >= a.keep_from) ? pol_last : pol_first;
+            uint4 r[2][NB];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int m = 0; m < NB; ++m)
+                    r[h][m] = have[m] ? ld16_policy(rowp[m] + e0 + 32 * h, pol) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    unsigned int lo[NB], hi[NB];
+#pragma unroll
+                    for (int m = 0; m < NB; ++m) {
+                        lo[m] = half ? r[h][m].z : r[h][m].x;
+                        hi[m] = half ? r[h][m].w : r[h][m].y;
+                    }
+#pragma unroll
+                    for (int cb = 0; cb < NB; ++cb)
+                        mma_bf16_16816_full(c[cb], lo[0], lo[1], hi[0], hi[1], lo[cb], hi[cb]);
+                }
+            chain += 4;
+            if (chain >= kMmaChain) {
+#pragma unroll
+                for (int i = 0; i < NT; ++i)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) { d[i][k] += (double)c[i][k]; c[i][k] = 0.f; }
+                chain = 0;
+            }
+        }
+    }
+    // the streaming part of this CTA is over: the finishing kernel may be placed (it waits for this grid)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < NT; ++i)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) wide_red[((size_t)(warp * NT + i) * 32 + lane) * 4 + k] = d[i][k] + (double)c[i][k];
+    __syncthreads();
+    const int tiles8 = NB;                           // 8 x 8 blocks per side
+    for (int e = threadIdx.x; e < NT * 128; e += kWideThreads) {
+        // the 16 warps in a fixed order
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) s += wide_red[(size_t)w * NT * 128 + e];
+        const int cb = e >> 7, ln = (e >> 2) & 31, k = e & 3;
+        const int bi = k >> 1, bj = cb;                                   // 8 x 8 block, row and column inside it:
+        const int row = ln >> 2, col = 2 * (ln & 3) + (k & 1);
+        if (bi > bj || bi >= tiles8) continue;                            // below the diagonal: not wanted
+        int tp = 0;
+        for (int q = 0; q < bi; ++q) tp += tiles8 - q;
+        tp += bj - bi;
+        a.partials[((size_t)tp * gridDim.x + blockIdx.x) * 64 + row * 8 + col] = s;
+    }
+    // ragged end (D mod 64 elements), first CTA: plain binary64 products, added to its own slots
+    const int64_t tail0 = n_tiles * kMmaTileElems;
+    if (blockIdx.x == 0 && tail0 < a.D) {
+        __syncthreads();
+        for (int p = threadIdx.x; p < a.K * a.K; p += kWideThreads) {
+            const int i = p / a.K, j = p % a.K;
+            if (i > j) continue;
+            const __nv_bfloat16 *xi = static_cast<const __nv_bfloat16 *>(a.g[i]), *xj = static_cast<const __nv_bfloat16 *>(a.g[j]);
+            double s = 0.0;
+            for (int64_t e = tail0; e < a.D; ++e) s += (double)load1<__nv_bfloat16>(xi, e) * (double)load1<__nv_bfloat16>(xj, e);
+            const int bi = i >> 3, bj = j >> 3;
+            int tp = 0;
+            for (int q = 0; q < bi; ++q) tp += tiles8 - q;
+            tp += bj - bi;
+            a.partials[((size_t)tp * gridDim.x + blockIdx.x) * 64 + (i & 7) * 8 + (j & 7)] += s;
+        }
+    }
+}
+
 }  // namespace gaf

@@ -165,7 +165,8 @@ def test_filter_maximum_k(ws, schedule):
 
 @pytest.mark.parametrize("K", [9, 16, 24, 32, 33, 48, 64])
 def test_filter_gram_first_on_tensor_cores(ws, K):
-    """bf16 with 9..64 gradients: the Gram matrix comes from the tcgen05 kernel."""
+    """bf16 with 9..64 gradients: the Gram matrix comes from the tensor cores -- warp-level MMAs fed from
+    the global loads up to 16 gradients (two blocks of 8 rows), the tcgen05 tile beyond."""
     w = _mix(K, 1_000_003 + 64 * K, "bf16", seed=200 + K)
     r = check_filter(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM)
     assert 1 < r["count"] < K
@@ -342,8 +343,8 @@ def test_bounded_waits_run_out_and_the_workspace_recovers(ws):
         # one-launch Gram-first schedule: the waiting CTAs are never shown the full arrival counter
         (_mix(4, 600_011, "f32", seed=11, rho=[0.8, 0.6, -0.2, 0.7]), gaf.GAF_SCHED_GRAM_FUSED),
         (_mix(8, 300_007, "bf16", seed=12), gaf.GAF_SCHED_GRAM_FUSED),
-        # tensor-core Gram pipeline: the first tile's barrier never completes
-        (_mix(16, 300_007, "bf16", seed=13), gaf.GAF_SCHED_GRAM),
+        # tcgen05 Gram pipeline (17..64 bfloat16 gradients): the first tile's barrier never completes
+        (_mix(17, 300_007, "bf16", seed=13), gaf.GAF_SCHED_GRAM),
         (_mix(40, 100_003, "bf16", seed=14), gaf.GAF_SCHED_GRAM),
     ]
     for w, schedule in cases:
@@ -514,7 +515,8 @@ def test_pairwise_small(ws, dtype):
 def test_pairwise_general_kernel_shapes(ws, dtype, K):
     """More than 8 gradients: the general CUDA-core Gram kernel (binary32) in each of its shapes (warps
     sharing a tile pair, one warp per pair, tile pairs split over groups of CTAs) and the tensor-core
-    kernel (bfloat16) in its 16-, 32- and 64-row forms: several panels or tiles per CTA, a ragged end."""
+    kernels (bfloat16: warp-level MMAs up to 16 gradients, the tcgen05 tile in its 32- and 64-row forms):
+    several panels or tiles per CTA, a ragged end."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     for D in (sms * 512 * 3 + 1234 + 3, 100_001):
         w = _mix(K, D, dtype, seed=300 + K)
@@ -544,6 +546,17 @@ def test_auto_schedule_choice(ws):
         g[i::8] = 1.0
     gaf.gaf_filter_accumulate(big, 0.97, ws)
     assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM and gaf.gaf_last_launch_count() == 2
+
+
+def test_wide_mma_gram_kernel_shapes_and_long_runs(ws):
+    """9..16 bfloat16 gradients (and the first counts of the tcgen05 tile behind them): absent rows feed zeros;
+    lengths below one tile, ragged ends, and a length from which the CTAs walk in runs of several trips."""
+    for K in (9, 12, 15, 16, 17, 24, 25):
+        for D in (37, 64 * 16 * 5 + 11, 300_001):
+            check_pairwise(_mix(K, D, "bf16", seed=700 + K).grads, ws)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    D = 32 * 8 * 16 * 64 * 2 * sms + 64 * 16 * 3 + 5      # just over the threshold for long runs
+    check_pairwise(_mix(12, D, "bf16", seed=777).grads, ws)
 
 
 def test_mma_gram_kernel_long_runs(ws):
