@@ -53,7 +53,7 @@ CONFIG_B = {1: 4, 2: 4, 3: 2, 4: 4, 5: 2}
 # and all sets together exceed L2 (configuration 1: 12 x 16 MB), so every call starts cold in L2
 N_SETS = {1: 12, 2: 4, 4: 2, 5: 1}
 # calls timed for the entries of the `configs` block
-BLOCK_STEPS = {1: 3000, 3: 300, 4: 100, 5: 60}
+BLOCK_STEPS = {1: 1000, 3: 300, 4: 100, 5: 60}
 
 
 def parse_args():
@@ -76,6 +76,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sets", type=int, default=None,
+                    help="number of rotating input sets of the headline workload (profiler captures: fewer sets, "
+                         "less device memory)")
     ap.add_argument("--no-configs", action="store_true",
                     help="leave out the `configs` block (the other named configurations)")
     return ap.parse_args()
@@ -113,16 +116,30 @@ def min_bytes(K, D, b):
     return (K * b + 4) * D
 
 
-# DRAM traffic (ncu dram__bytes_read.sum + dram__bytes_write.sum, per launch, summed over the launches
-# of a call) of the kernels as committed, taken from the captures that the summaries in the profiler
-# folder of this repository describe.  Bytes per element index and accepted count c; a capture on a
-# shorter vector of the same recipe scales in proportion (both passes stream).  An entry is used only
-# while the listed kernel sources hash to what was profiled; otherwise `traffic` is null.
+# DRAM traffic (ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, summed over the launches of a
+# call) of the kernels as committed, from the captures that the summaries in the profiler folder of this
+# repository describe.  Bytes per element index, by accepted count c.  Two captures per entry where they differ:
+#   "steady"   caches left as the previous call left them (ncu --cache-control none): what crosses HBM while
+#              calls run back to back, as they do in the timed region -- this is `traffic`;
+#   "flushed"  ncu's default, caches flushed before every launch: a call that starts with a cold L2.
+# At configuration 2 they differ: back to back, about 32 MB of L2 hold the previous call's output (dirty lines
+# that the next call overwrites in place, so they never reach HBM) and fewer of the second pass's re-reads hit.
+# Captures on a shorter vector of the same recipe scale in proportion (both passes stream; inputs far beyond
+# L2).  An entry is used only while the listed kernel sources hash to what was profiled; otherwise null.
 NCU_TRAFFIC = {
     # gram_fused_kernel<float,4> at configuration 2 itself (D = 11,227,812)
     (2, 3): {"sources": ["gaf_fused.cuh", "gaf_gramfilter.cuh", "gaf_device.cuh"],
-             "sha256": "",
-             "bytes_per_element": {}},
+             "sha256": "b0251f16d69b2f78f384133653cd9c83ffea9080495cada25e29c219c1acb77f",
+             "steady": {2: 262.7e6 / 11227812, 3: 296.6e6 / 11227812},
+             "flushed": {2: 232.0e6 / 11227812, 3: 259.6e6 / 11227812}},
+    # gram_small_kernel<float,8> + masked_mean_kernel<float>, captured at D = 80,000,000
+    (4, 2): {"sources": ["gaf_gramfilter.cuh", "gaf_device.cuh"],
+             "sha256": "605c2ef6d0cc865bb09a5d25d703927c4c13c9bf97bcbaca7df1d0e48b9c36f9",
+             "steady": {4: (2563.4e6 + 1573.8e6) / 80e6, 1: (2563.9e6 + 590.8e6) / 80e6}},
+    # gram_mma_kernel<8> + masked_mean_kernel<bf16>, captured at D = 100,000,000
+    (5, 2): {"sources": ["gaf_gram_mma.cuh", "gaf_gramfilter.cuh", "gaf_device.cuh"],
+             "sha256": "86fbf6b03aea3b7b91bdaebc2b2fbc16cf23a7bb73634aaa93d0f7cd31c310c4",
+             "steady": {4: (1604.2e6 + 1170.1e6) / 100e6}},
 }
 
 
@@ -135,13 +152,13 @@ def kernel_sources_hash(names):
     return h.hexdigest()
 
 
-def ncu_traffic(cfg, sched_used, masks, D, n_sets, steps):
+def ncu_traffic(cfg, sched_used, masks, D, n_sets, steps, which="steady"):
     """Average DRAM bytes per call over the rotating input sets, or None when no capture of the
     committed kernels is on record for this configuration and schedule."""
     entry = NCU_TRAFFIC.get((cfg, sched_used))
     if not entry or kernel_sources_hash(entry["sources"]) != entry["sha256"]:
         return None
-    table = entry["bytes_per_element"]
+    table = entry.get(which) or entry["steady"]
     per_set = []
     for m in masks:
         c = sum(int(x) for x in m)
@@ -391,20 +408,21 @@ def timed_region(torch, step, steps, warmup, nvml, barrier=None, ramp_seconds=RA
             "clocks": clocks, "per_call_ms": per_call}
 
 
-def fractions(ms, traffic, model_b, min_b, peak):
+def fractions(ms, traffic, model_b, min_b, peak, traffic_flushed=None):
     """The three byte counts over one time, as GB/s and as fractions of `peak`."""
     def rate(nbytes):
         return None if nbytes is None else nbytes / (ms * 1e-3) / 1e9
-    dram, model, least = rate(traffic), rate(model_b), rate(min_b)
+    dram, model, least, cold = rate(traffic), rate(model_b), rate(min_b), rate(traffic_flushed)
     return {"dram_gbs": dram, "dram_frac": None if dram is None else dram / peak,
+            "dram_frac_flushed_caches": None if cold is None else cold / peak,
             "model_gbs": model, "model_frac": model / peak,
             "min_bytes_gbs": least, "min_bytes_frac": least / peak}
 
 
 def measure_filter(torch, gaf, workloads, cfg, dev, tau, schedule, steps, warmup, nvml, rank=0, D=None,
-                   barrier=None, want_warm=False, want_c_loop=False):
+                   barrier=None, want_warm=False, want_c_loop=False, n_sets=None):
     """One named configuration of the filter on one GPU: timed region, byte counts, fractions."""
-    n_sets = N_SETS[cfg]
+    n_sets = n_sets or N_SETS[cfg]
     sets = [workloads.config(cfg, device=dev, seed=(cfg - 1) + 1000 * i + 17 * rank, D=D) for i in range(n_sets)]
     w0 = sets[0]
     K, D, b = w0.K, w0.D, w0.elem_bytes
@@ -440,6 +458,8 @@ def measure_filter(torch, gaf, workloads, cfg, dev, tau, schedule, steps, warmup
            "sched_used": sched_used, "launches_per_step": launches_per_step, "status": status,
            "model_bytes": model_b, "min_bytes": min_bytes(K, D, b),
            "traffic": ncu_traffic(cfg, sched_used, masks, D, n_sets, steps) if abs(tau - 0.97) < 1e-12 else None,
+           "traffic_flushed": (ncu_traffic(cfg, sched_used, masks, D, n_sets, steps, "flushed")
+                               if abs(tau - 0.97) < 1e-12 else None),
            "timing": t, "sets": sets, "ws": ws, "outputs": (macro, mask, dist_out, count), "dtype_code": dtype_code}
 
     if want_warm:
@@ -479,7 +499,7 @@ def block_entry(m, peak, peak_kind, tau, schedule):
     """One entry of the `configs` block from a measure_filter result."""
     t = m["timing"]
     ms = t["ms_per_step"]
-    fr = fractions(ms, m["traffic"], m["model_bytes"], m["min_bytes"], peak)
+    fr = fractions(ms, m["traffic"], m["model_bytes"], m["min_bytes"], peak, m["traffic_flushed"])
     per_call = t["per_call_ms"]
     mhz = t["clocks"]["sm_mhz"]
     e = {"workload": workload_label(m["cfg"], m["K"], m["D"], m["dtype"], tau),
@@ -602,12 +622,13 @@ def run_ours(args):
     cfg, steps = args.workload, args.steps
     peak, peak_kind = peak_bandwidth()
     m = measure_filter(torch, gaf, workloads, cfg, dev, args.tau, args.schedule, steps, args.warmup, nvml,
-                       rank=rank, D=args.D, barrier=barrier, want_warm=cfg in (1, 2), want_c_loop=True)
+                       rank=rank, D=args.D, barrier=barrier, want_warm=cfg in (1, 2), want_c_loop=True,
+                       n_sets=args.sets)
     t = m["timing"]
     K, D, b, grad_bytes = m["K"], m["D"], m["b"], m["grad_bytes"]
     ms_per_step = max_over_ranks(t["ms_region"], dev) / steps
     value = aggregate_gbs(world, grad_bytes, ms_per_step)
-    fr = fractions(ms_per_step, m["traffic"], m["model_bytes"], m["min_bytes"], peak)
+    fr = fractions(ms_per_step, m["traffic"], m["model_bytes"], m["min_bytes"], peak, m["traffic_flushed"])
     per_call = t["per_call_ms"]
 
     # end to end through the host-buffer entry point
@@ -692,10 +713,12 @@ def run_ours(args):
                  **({"note": "REDUCED length, not the named configuration"} if args.D else {})}),
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "basis": ("dram: bytes that crossed HBM per call (ncu, `traffic`) / time" if basis == "dram" else
+                "basis": ("dram: bytes that cross HBM per call while calls run back to back (ncu --cache-control none, "
+                          "`traffic`) / time; dram_frac_flushed_caches takes ncu's default capture (caches flushed "
+                          "before the launch) instead" if basis == "dram" else
                           "min_bytes: (K b + 4) D / time (no DRAM traffic on record for the kernels as committed)"),
-                "traffic": m["traffic"], "peak_kind": peak_kind,
-                "dram_frac": fr["dram_frac"], "min_bytes_frac": fr["min_bytes_frac"], "model_frac": fr["model_frac"],
+                "traffic": m["traffic"], "traffic_flushed_caches": m["traffic_flushed"], "peak_kind": peak_kind,
+                "dram_frac": fr["dram_frac"], "dram_frac_flushed_caches": fr["dram_frac_flushed_caches"], "min_bytes_frac": fr["min_bytes_frac"], "model_frac": fr["model_frac"],
                 "dram_gbs": fr["dram_gbs"], "min_bytes_gbs": fr["min_bytes_gbs"], "model_gbs": fr["model_gbs"],
                 "frac_of_nominal_8000": achieved / 8000.0,
                 "kernel": {3: "gram_fused_kernel (the whole call is this one launch)",
