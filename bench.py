@@ -336,7 +336,8 @@ def run_reference(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
         "config": config_dict(cfg, K, full, w.dtype, args.tau, "CPU oracle (Algorithm 1 as written, one thread)",
-                              "host cores", f"each step runs on D={w.D} elements of the recipe"),
+                              "host cores", f"each step runs on D={w.D} elements of the recipe",
+                              {"accept_masks": None}),
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,

@@ -18,17 +18,25 @@
  *     what lives in the caller's workspace.
  *   - Every call is asynchronous on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and never synchronises, except
- *     gaf_read_status and the *_host convenience call, which say so.
+ *     gaf_read_status and the *_host convenience call, which say so.  Some
+ *     kernels are launched with programmatic stream serialisation and signal
+ *     early that the launch behind them may be placed: an ordinary launch
+ *     behind a call is ordered after it as usual; a launch that the caller
+ *     itself makes programmatic must, as always with such launches, wait for
+ *     its predecessor (griddepcontrol.wait / cudaGridDependencySynchronize)
+ *     before it reads the call's outputs.
  *   - Gradient buffers are read-only.  Every device pointer must be 16-byte
  *     aligned (else GAF_ERR_ALIGN).  D need not be a multiple of anything; with
  *     D == 0 the element buffers may be NULL.
  *   - dtype: GAF_F32 = IEEE binary32, GAF_BF16 = bfloat16.  Arithmetic on
- *     elements is binary32 (products of at most 64 pairs are summed in binary32
- *     before they are widened; the Gram sums of up to 4 binary32 gradients are
- *     taken in binary64 throughout, where every product is exact); sums are
- *     carried in binary64 from the thread level up and reduced in a fixed
- *     order, so results are bitwise reproducible on the same GPU model.  The
- *     scalar arithmetic of Eq. 4 and the comparison with tau are binary64.
+ *     elements is binary32: products of at most 64 pairs are summed in binary32
+ *     before they are widened (on the tensor-core paths that bfloat16 gradients
+ *     take from 7 gradients on: binary32 accumulators over at most 512 products);
+ *     the Gram sums of up to 4 binary32 gradients are taken in binary64
+ *     throughout, where every product is exact.  Sums are carried in binary64
+ *     from the thread level up and reduced in a fixed order, so results are
+ *     bitwise reproducible on the same GPU model.  The scalar arithmetic of
+ *     Eq. 4 and the comparison with tau are binary64.
  *   - Conventions where the paper is silent: a pair with a zero-norm member has
  *     cos := 0 (distance 1); cos is clamped to [-1, 1]; a NaN distance is
  *     rejected.  Either event sets a bit in the status word (see

@@ -87,6 +87,21 @@ def test_filter_argument_errors(L):
     assert _filter(L, g, 4, 100, ws_bytes=100) == 4
 
 
+def test_repeat_and_test_hook_argument_errors(L):
+    g = [A + i * (1 << 24) for i in range(8)]
+    arr = (ctypes.c_void_p * 8)(*g)
+    p = ctypes.cast(arr, ctypes.c_void_p)
+    out, mask, count, ws = A + (1 << 30), A + (2 << 30), A + (3 << 30), A + (4 << 30)
+
+    def rep(repeats, n_sets, K, grads=p, workspace=ws):
+        return L.gaf_filter_accumulate_repeat(repeats, n_sets, grads, K, 100, 0, 0.97, None, out, mask, None, count,
+                                              workspace, 1 << 22, 0, None)
+    assert rep(-1, 2, 4) == 1 and rep(3, 0, 4) == 1 and rep(3, 2, 0) == 1 and rep(3, 2, 4, grads=None) == 1
+    assert rep(0, 2, 4) == 0                        # no repetition: nothing is launched, nothing is checked further
+    assert rep(2, 2, 4, workspace=0) == 4           # the first repetition's own checks apply
+    assert L.gaf_test_set_wait_fault(1000, 1) == 0 and L.gaf_test_set_wait_fault(0, 0) == 0
+
+
 def test_cosdist_and_pairwise_argument_errors(L):
     ws, n = A + (4 << 30), 1 << 22
     assert L.gaf_cosdist(None, A, 10, 0, A + 4096, None, ws, n, None) == 1

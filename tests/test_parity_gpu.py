@@ -217,6 +217,25 @@ def test_filter_host_entry_point(ws):
     assert torch.equal(dist.cpu(), dist_h) and int(count.item()) == int(count_h.item())
 
 
+def test_repeat_entry_point(ws):
+    """gaf_filter_accumulate_repeat is a host loop in C around gaf_filter_accumulate: after r calls over
+    rotating input sets the outputs are those of the last set used, and the launches add up."""
+    sets = [_mix(4, 200_003, "f32", seed=70 + i, rho=[0.8, 0.6, -0.2, 0.7] if i else [0.7, -0.3, 0.5, 0.1]).grads
+            for i in range(3)]
+    D = 200_003
+    macro = torch.empty(D, device="cuda"); mask = torch.empty(4, dtype=torch.uint8, device="cuda")
+    dist = torch.empty(4, device="cuda"); count = torch.empty(1, dtype=torch.int32, device="cuda")
+    for repeats in (1, 3, 5):
+        gaf.gaf_filter_accumulate_repeat(repeats, sets, 0.9, ws, macro, mask, dist, count)
+        launches = gaf.gaf_last_launch_count()
+        want = gaf.gaf_filter_accumulate(sets[(repeats - 1) % 3], 0.9, ws)
+        assert launches == repeats * gaf.gaf_last_launch_count()
+        assert torch.equal(macro, want[0]) and torch.equal(mask, want[1])
+        assert torch.equal(dist, want[2]) and torch.equal(count, want[3])
+    gaf.gaf_filter_accumulate_repeat(0, sets, 0.9, ws, macro, mask, dist, count)     # nothing to do is legal
+    assert gaf.gaf_last_launch_count() == 0
+
+
 def test_filter_random_cases(ws):
     """Seeded random shapes, thresholds, orders and schedules against the oracle."""
     rng = np.random.RandomState(2024)
