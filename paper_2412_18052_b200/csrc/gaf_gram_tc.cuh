@@ -15,14 +15,16 @@
 // ignored.
 //
 // Pipeline per CTA (one CTA per SM; tiles of the D axis are dealt round-robin to the CTAs):
-//   warps 4-7  loaders: 16-byte cp.async copies global -> swizzled shared memory, a ring of
-//              kTcStages tiles of 16 KB, each copy batch arriving on the tile's mbarrier by itself;
-//   warp 8     one thread issues the MMAs (4 per tile, K = 16 each) into one of two
+//   warps 4-11 loaders: 16-byte cp.async copies global -> swizzled shared memory, a ring of
+//              kTcStages tiles of 64 KB, each copy batch arriving on the tile's mbarrier by itself;
+//   warp 12    one thread issues the MMAs (16 per tile, K = 16 each) into one of two
 //              128-column accumulator buffers in tensor memory and commits to mbarriers;
 //   warps 0-3  epilogue: every kTcDrain tiles read the finished buffer with tcgen05.ld and
 //              add it to binary64 registers (short binary32 accumulation chains only).
 // A tile is kTcSub swizzle blocks (kTcSub x 64 elements per row): the issuing thread pays
-// one barrier handshake per tile, which at one block per tile cost more than the MMAs.
+// one barrier handshake per tile, which at one block per tile cost more than the MMAs.  Measured
+// at 32 gradients, D = 11.2 M, in a long loop of calls: six tiles of two blocks 139-149 us, three tiles of
+// four blocks 125-134 us (fewer, larger handshakes; 64 gradients: 289 -> 252 us).
 // At the end the R chunk blocks are summed in a fixed order and the CTA writes its partial
 // Gram matrix in the [tile pair][slice][64] layout of the CUDA-core version, so the same
 // finishing kernel totals the slices.  Every wait is bounded.
@@ -36,10 +38,10 @@ namespace gaf {
 #define GAF_TC_LOADER_WARPS 8
 #endif
 #ifndef GAF_TC_STAGES
-#define GAF_TC_STAGES 6
+#define GAF_TC_STAGES 3
 #endif
 #ifndef GAF_TC_SUB
-#define GAF_TC_SUB 2
+#define GAF_TC_SUB 4
 #endif
 constexpr int kTcLoaderWarps = GAF_TC_LOADER_WARPS;
 constexpr int kTcLoaders = kTcLoaderWarps * 32;
