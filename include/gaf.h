@@ -67,7 +67,8 @@ enum {
     GAF_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or too small */
     GAF_ERR_CUDA = 5,           /* a CUDA runtime call failed (launch, copy) */
     GAF_ERR_RESERVED = 6,       /* not used */
-    GAF_ERR_UNSUPPORTED = 7,    /* the requested schedule cannot run on this device */
+    GAF_ERR_UNSUPPORTED = 7,    /* the requested schedule cannot run for this call (K too large for it, or the
+                                   device is still busy with a one-launch call on another stream) */
     GAF_ERR_TOO_LARGE = 8       /* size beyond the fixed limit of gaf_cosdist_static */
 };
 
@@ -97,9 +98,13 @@ enum {
                                    itself from the partial sums all CTAs left in the workspace, so that
                                    part of what the first pass read (shared memory, L2) need not cross
                                    HBM again.  Identical outputs to GAF_SCHED_GRAM.  GAF_ERR_UNSUPPORTED
-                                   for K > 8.  Its one wait on other CTAs is bounded:
-                                   GAF_STATUS_TIMEOUT if it ever runs out (it can only run out when
-                                   something else keeps part of the device busy for seconds). */
+                                   for K > 8.  Such a call needs the whole device for its CTAs to meet:
+                                   calls on one stream are ordered and fine; a second one on ANOTHER
+                                   stream while the first stream still has work pending returns
+                                   GAF_ERR_UNSUPPORTED (GAF_SCHED_AUTO takes two launches then).  The one
+                                   wait on other CTAs is bounded: GAF_STATUS_TIMEOUT if it ever runs out
+                                   (only when something else, another process say, keeps part of the
+                                   device busy for seconds). */
 };
 
 /* Bits of the device status word. */

@@ -355,6 +355,18 @@ constexpr int kParkBytesPerSm = 128 << 10;
 constexpr int64_t kFusedMaxInputBytesF32 = int64_t(512) << 20;
 constexpr int64_t kFusedMaxInputBytesBf16Mma = int64_t(1) << 30;
 
+// A one-launch call needs the whole device: its CTAs wait for one another, so two such grids in flight at once
+// (two streams) could each hold part of the SMs and wait for the rest until their bounded waits run out.  Calls on
+// one stream are ordered and safe.  The library therefore remembers, per device, the stream of its latest
+// one-launch call, and refuses another one on a DIFFERENT stream while that stream still has work pending
+// (GAF_ERR_UNSUPPORTED: the library's own choice then takes the two-launch form, which has no such need).
+struct FusedGuard {
+    std::mutex m;
+    cudaStream_t last = nullptr;
+    bool any = false;
+};
+FusedGuard g_fused_guard[kMaxDevices];
+
 template <typename T, int KT>
 int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st) {
     auto kernel = gram_fused_kernel<T, KT>;
@@ -408,6 +420,13 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
     // resident and the one wait on other CTAs ends; it is bounded in any case.  Programmatic stream
     // serialisation: the kernel waits for its predecessor on the stream itself (griddepcontrol.wait, first
     // thing) and releases its successor once its decisions are taken.
+    FusedGuard &guard = g_fused_guard[di.dev];
+    std::lock_guard<std::mutex> lock(guard.m);          // (check and launch are one step for other host threads)
+    if (guard.any && guard.last != st) {
+        const cudaError_t q = cudaStreamQuery(guard.last);
+        if (q == cudaErrorNotReady) return GAF_ERR_UNSUPPORTED;
+        if (q != cudaSuccess) cudaGetLastError();       // that stream no longer exists: nothing of it is in flight
+    }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(unsigned(grid)); cfg.blockDim = dim3(kGsThreads);
     cfg.dynamicSmemBytes = size_t(pl.dyn); cfg.stream = st;
@@ -417,6 +436,8 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
     cfg.attrs = attr; cfg.numAttrs = 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, a);
     if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+    guard.last = st;
+    guard.any = true;
     ++g_launches;
     return GAF_OK;
 }
@@ -594,7 +615,7 @@ const char *gaf_error_string(int code) {
         case GAF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case GAF_ERR_CUDA: return "CUDA runtime error";
         case GAF_ERR_RESERVED: return "reserved";
-        case GAF_ERR_UNSUPPORTED: return "schedule not supported on this device";
+        case GAF_ERR_UNSUPPORTED: return "schedule not available for this call on this device";
         case GAF_ERR_TOO_LARGE: return "size beyond the fixed limit of the no-allocation entry point";
         default: return "unknown error code";
     }

@@ -236,6 +236,39 @@ def test_repeat_entry_point(ws):
     assert gaf.gaf_last_launch_count() == 0
 
 
+def test_one_launch_calls_do_not_overlap_across_streams(ws):
+    """A one-launch call needs the whole device.  While one is in flight on a stream, an explicit request on
+    another stream is refused and the library's own choice takes two launches; ordered on one stream, or once
+    the first stream is idle, the one-launch form runs again.  Results are correct throughout."""
+    w = _mix(4, 30_000_011, "f32", seed=88, rho=[0.8, 0.6, -0.2, 0.7])       # a call of about 150 us
+    small = _mix(4, 100_003, "f32", seed=89, rho=[0.8, 0.6, -0.2, 0.7])
+    ws2 = gaf.new_workspace(4, 1 << 20, gaf.GAF_F32)
+    want = [t.clone() for t in gaf.gaf_filter_accumulate(small.grads, 0.9, ws2, schedule=gaf.GAF_SCHED_GRAM)]
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    refused = fell_back = 0
+    for _ in range(5):
+        with torch.cuda.stream(s1):
+            for _ in range(4):
+                gaf.gaf_filter_accumulate(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED)   # same stream: fine
+        with torch.cuda.stream(s2):
+            try:
+                gaf.gaf_filter_accumulate(small.grads, 0.9, ws2, schedule=gaf.GAF_SCHED_GRAM_FUSED)
+            except gaf.GafError as e:
+                assert e.code == 7
+                refused += 1
+            got = gaf.gaf_filter_accumulate(small.grads, 0.9, ws2)            # AUTO: whatever may run now
+            fell_back += gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM
+        torch.cuda.synchronize()
+        for x, y in zip(got, want):
+            assert torch.equal(x, y)
+    assert refused >= 1 and fell_back >= 1          # (0.6 ms of work was pending on the first stream each time)
+    with torch.cuda.stream(s2):
+        gaf.gaf_filter_accumulate(small.grads, 0.9, ws2, schedule=gaf.GAF_SCHED_GRAM_FUSED)      # first stream idle: fine
+    torch.cuda.synchronize()
+    check_filter(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED)
+
+
 def test_filter_random_cases(ws):
     """Seeded random shapes, thresholds, orders and schedules against the oracle."""
     rng = np.random.RandomState(2024)
