@@ -542,6 +542,32 @@ def measure_pairwise(torch, gaf, workloads, dev, steps, warmup, nvml, K=None, D=
                        "gram_panel_kernel" if K > 8 else "gram_small_kernel") + " + finishing (whole call)"}
 
 
+def measure_cosdist(torch, gaf, workloads, dev, D, steps, nvml, peak, peak_kind):
+    """gaf_cosdist (Eq. 4 between two buffers) on two gradients of configuration 2's recipe at length D."""
+    w = workloads.config(2 if D == FULL_D[2] else 4, device=dev, K=2, D=D)
+    ws = gaf.new_workspace(2, D, gaf.GAF_F32, device=dev)
+    dist_out = torch.empty(1, dtype=torch.float32, device=dev)
+    stats = torch.empty(3, dtype=torch.float64, device=dev)
+    n_sets = 4 if 2 * 4 * D * 4 < 4e9 else 1
+    pairs = [w.grads] + [[g.clone() for g in w.grads] for _ in range(n_sets - 1)]
+
+    def step(i):
+        x, y = pairs[i % n_sets]
+        gaf.gaf_cosdist(x, y, ws, dist_out=dist_out, stats_out=stats)
+
+    t = timed_region(torch, step, steps, 5, nvml)
+    ms = t["ms_per_step"]
+    nbytes = 2 * 4 * D
+    rate = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": f"gaf_cosdist, D={D}, f32 inputs ({n_sets} rotating pairs of {nbytes / 1e6:.0f} MB)",
+            "op": "gaf_cosdist", "steps": steps, "ramp_calls": t["ramp_calls"], "ms_per_call": ms,
+            "ms_per_call_median_of_event_pairs": statistics.median(t["per_call_ms"]), "value": rate, "unit": UNIT,
+            "launches_per_call": 1, "min_bytes_per_call": nbytes, "model_bytes_per_call": nbytes,
+            "byte_model": "both buffers read once: 2 b D (= the minimum)", "min_bytes_frac": rate / peak,
+            "model_frac": rate / peak, "dram_frac": None, "traffic": None, "peak": peak, "peak_kind": peak_kind,
+            "clocks": t["clocks"]}
+
+
 def pairwise_entry(m, peak, peak_kind, steps):
     t = m["timing"]
     ms = t["ms_per_step"]
@@ -684,6 +710,13 @@ def run_ours(args):
             except Exception as exc:      # a configuration that cannot run here is reported, not hidden
                 block[str(c)] = {"error": f"{type(exc).__name__}: {exc}"}
             r = None
+            gc.collect()
+            torch.cuda.empty_cache()
+        for key, D_c, n in (("cosdist_D11.2M", FULL_D[2], 1000), ("cosdist_D124M", FULL_D[4], 200)):
+            try:
+                block[key] = measure_cosdist(torch, gaf, workloads, dev, D_c, n, nvml, peak, peak_kind)
+            except Exception as exc:
+                block[key] = {"error": f"{type(exc).__name__}: {exc}"}
             gc.collect()
             torch.cuda.empty_cache()
 

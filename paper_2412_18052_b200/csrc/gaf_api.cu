@@ -659,8 +659,10 @@ int gaf_cosdist(const void *x, const void *y, int64_t D, int dtype, float *dist_
               reinterpret_cast<double *>(base + kPartialsOffset), dist_out, stats_out};
     const int grid = stream_grid(D, kStepThreads, di.sms);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (dtype == GAF_F32) cosdist_kernel<float><<<grid, kStepThreads, 0, st>>>(a);
-    else cosdist_kernel<__nv_bfloat16><<<grid, kStepThreads, 0, st>>>(a);
+    // (the kernel waits for its predecessor on the stream itself and releases its successor when its streaming part ends)
+    const cudaError_t err = dtype == GAF_F32 ? launch_dependent(cosdist_kernel<float>, grid, kStepThreads, st, a)
+                                             : launch_dependent(cosdist_kernel<__nv_bfloat16>, grid, kStepThreads, st, a);
+    if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? GAF_OK : GAF_ERR_CUDA;
 }

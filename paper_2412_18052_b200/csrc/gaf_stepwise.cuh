@@ -165,6 +165,9 @@ __global__ void __launch_bounds__(kStepThreads, 2) cosdist_kernel(CosArgs a) {
     __shared__ bool is_last;
     const T *x = static_cast<const T *>(a.x);
     const T *y = static_cast<const T *>(a.y);
+    // launched with programmatic stream serialisation by gaf_cosdist: nothing the launch before it on the stream
+    // wrote is touched before that launch has completed (a no-op after an ordinary predecessor or launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (blockIdx.x == 0 && threadIdx.x == 0) a.ctl->status = 0;
 
     Sums3 s = {0.0, 0.0, 0.0};
@@ -186,6 +189,8 @@ __global__ void __launch_bounds__(kStepThreads, 2) cosdist_kernel(CosArgs a) {
         s.na += (double)(xv * xv);
         s.ng += (double)(yv * yv);
     }
+    // the streaming part of this CTA is over: the launch behind this one may be placed (it waits for this grid)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     Sums3 blk = block_reduce(s, scratch);
     if (threadIdx.x == 0) {
         a.partials[3 * blockIdx.x] = blk.p;
