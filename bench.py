@@ -70,6 +70,8 @@ def parse_args():
                          "the line then says so in config.workload")
     ap.add_argument("--K", type=int, default=None, help="pairwise workload only: another number of gradients")
     ap.add_argument("--fp32", action="store_true", help="pairwise workload only: binary32 inputs (same recipe)")
+    ap.add_argument("--separate", action="store_true",
+                    help="pairwise workload only: K separate allocations instead of the rows of one matrix")
     ap.add_argument("--tau", type=float, default=0.97)
     ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2, 3],
                     help="0 auto, 1 stepwise (streaming), 2 Gram-first in two launches, 3 Gram-first in one launch")
@@ -521,11 +523,13 @@ def block_entry(m, peak, peak_kind, tau, schedule):
     return e
 
 
-def measure_pairwise(torch, gaf, workloads, dev, steps, warmup, nvml, K=None, D=None, fp32=False):
-    """Configuration 3: the K x K pairwise cosine-distance matrix."""
-    w = workloads.config(3, device=dev, K=K, D=D)
+def measure_pairwise(torch, gaf, workloads, dev, steps, warmup, nvml, K=None, D=None, fp32=False, stacked=True):
+    """Configuration 3: the K x K pairwise cosine-distance matrix.  ``stacked``: the gradients are the rows of one
+    matrix (row distance D rounded up to 128 elements: what an all-gather of padded flat micro-gradients leaves), which
+    lets the tensor-memory kernel fetch them by tensor copies; otherwise K separate allocations."""
+    w = workloads.config(3, device=dev, K=K, D=D, stacked=stacked)
     if fp32:
-        w = workloads.mixture(w.K, w.D, "f32", w.rho, w.seed, device=dev)
+        w = workloads.mixture(w.K, w.D, "f32", w.rho, w.seed, device=dev, stacked=stacked)
     K, D, b = w.K, w.D, w.elem_bytes
     ws = gaf.new_workspace(K, D, gaf.GAF_F32 if fp32 else gaf.GAF_BF16, device=dev)
     dist_out = torch.empty(K, K, dtype=torch.float32, device=dev)
@@ -536,9 +540,13 @@ def measure_pairwise(torch, gaf, workloads, dev, steps, warmup, nvml, K=None, D=
 
     step(0)
     launches = gaf.gaf_last_launch_count()
+    loader = gaf.gaf_last_gram_loader()
     t = timed_region(torch, step, steps, warmup, nvml)
     return {"K": K, "D": D, "b": b, "dtype": w.dtype, "grad_bytes": K * b * D, "launches": launches, "timing": t,
-            "kernel": ("gram_tc_kernel" if (not fp32 and 8 < K <= 64) else
+            "placement": "rows of one matrix" if stacked else "separate allocations",
+            "gram_loader": {0: None, 1: "16-byte asynchronous copies", 2: "tensor copies (TMA)"}[loader],
+            "kernel": ("gram_tc_kernel" if (not fp32 and 16 < K <= 64) else
+                       "gram_mma_wide_kernel" if (not fp32 and 8 < K <= 16) else
                        "gram_panel_kernel" if K > 8 else "gram_small_kernel") + " + finishing (whole call)"}
 
 
@@ -577,7 +585,8 @@ def pairwise_entry(m, peak, peak_kind, steps):
             "op": "gaf_pairwise_cosdist", "steps": steps, "ramp_calls": t["ramp_calls"], "ms_per_call": ms,
             "ms_per_call_median_of_event_pairs": statistics.median(t["per_call_ms"]),
             "event_pairs": len(t["per_call_ms"]), "value": achieved, "unit": UNIT,
-            "launches_per_call": m["launches"], "kernel": m["kernel"],
+            "launches_per_call": m["launches"], "kernel": m["kernel"], "placement": m["placement"],
+            "gram_loader": m["gram_loader"],
             "l2": f"inputs of one call ({m['grad_bytes'] / 1e6:.0f} MB) exceed the 126 MB L2",
             "model_bytes_per_call": m["grad_bytes"], "min_bytes_per_call": m["grad_bytes"],
             "byte_model": "every gradient read once: K b D (= the minimum)",
@@ -602,7 +611,7 @@ def run_pairwise(args):
     nvml = Nvml(0)
     named = args.K is None and args.D is None and not args.fp32
     m = measure_pairwise(torch, gaf, workloads, "cuda:0", args.steps, args.warmup, nvml, K=args.K, D=args.D,
-                         fp32=args.fp32)
+                         fp32=args.fp32, stacked=not args.separate)
     peak, peak_kind = peak_bandwidth()
     e = pairwise_entry(m, peak, peak_kind, args.steps)
     K = m["K"]
@@ -613,7 +622,7 @@ def run_pairwise(args):
         "dtype": "f32 products, f64 sums" if (args.fp32 or K > 64) else "bf16 x bf16 -> f32 (tensor cores), f64 sums",
         "data": "synthetic",
         "config": {"workload": e["workload"] + ("" if named else " (NOT the named configuration: size or type overridden)"),
-                   "K": K, "D": m["D"], "l2": e["l2"]},
+                   "K": K, "D": m["D"], "l2": e["l2"], "placement": m["placement"], "gram_loader": m["gram_loader"]},
         "roofline": {"bound": "hbm", "achieved": e["value"], "peak": peak, "unit": "GB/s", "frac": e["value"] / peak,
                      "basis": "min_bytes (= byte model: every gradient read once)", "traffic": None,
                      "peak_kind": peak_kind, "kernel": m["kernel"], "algorithmic_bytes_per_launch": m["grad_bytes"],
@@ -702,6 +711,14 @@ def run_ours(args):
                 if c == 3:
                     r = measure_pairwise(torch, gaf, workloads, dev, BLOCK_STEPS[3], 5, nvml)
                     block["3"] = pairwise_entry(r, peak, peak_kind, BLOCK_STEPS[3])
+                    r = None
+                    gc.collect()
+                    torch.cuda.empty_cache()
+                    r = measure_pairwise(torch, gaf, workloads, dev, BLOCK_STEPS[3], 5, nvml, stacked=False)
+                    other = pairwise_entry(r, peak, peak_kind, BLOCK_STEPS[3])
+                    block["3"]["separate_allocations"] = {k: other[k] for k in (
+                        "placement", "gram_loader", "ms_per_call", "ms_per_call_median_of_event_pairs", "value",
+                        "min_bytes_frac", "ms_x_sm_mhz")}
                 else:
                     r = measure_filter(torch, gaf, workloads, c, dev, 0.97, 0, BLOCK_STEPS[c], 5, nvml,
                                        want_warm=(c == 1), want_c_loop=(c == 1))

@@ -25,7 +25,7 @@ EXPORTS = [
     "gaf_filter_accumulate", "gaf_host_staging_bytes", "gaf_filter_accumulate_host",
     "gaf_pairwise_cosdist", "gaf_read_status", "gaf_last_launch_count", "gaf_cosdist_static",
     "gaf_filter_accumulate_any_seed", "gaf_stream_begin", "gaf_stream_push", "gaf_stream_end",
-    "gaf_filter_accumulate_bucketed", "gaf_last_schedule", "gaf_test_set_wait_fault",
+    "gaf_filter_accumulate_bucketed", "gaf_last_schedule", "gaf_last_gram_loader", "gaf_test_set_wait_fault",
     "gaf_filter_accumulate_repeat",
 ]
 
@@ -62,6 +62,7 @@ def lib() -> ctypes.CDLL:
         L.gaf_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.gaf_last_launch_count.argtypes = []
         L.gaf_last_schedule.argtypes = []
+        L.gaf_last_gram_loader.argtypes = []
         L.gaf_test_set_wait_fault.argtypes = [ctypes.c_uint, i32]
         L.gaf_cosdist_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
         L.gaf_filter_accumulate_any_seed.argtypes = [vp, i32, i64, i32, dbl, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -325,6 +326,12 @@ def gaf_last_launch_count() -> int:
 def gaf_last_schedule() -> int:
     """The GAF_SCHED_* value the latest gaf_filter_accumulate call of this thread ran with."""
     return lib().gaf_last_schedule()
+
+
+def gaf_last_gram_loader() -> int:
+    """How the tensor-memory Gram kernel of this thread's latest call fetched its tiles: 0 not used,
+    1 16-byte copies, 2 tensor copies (gradients that are rows of one matrix)."""
+    return lib().gaf_last_gram_loader()
 
 
 def gaf_test_set_wait_fault(wait_limit: int, withhold: bool) -> None:

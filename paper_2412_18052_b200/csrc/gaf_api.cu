@@ -31,6 +31,7 @@ thread_local int g_schedule = 0;       // what the latest gaf_filter_accumulate 
 // Test hook (gaf_test_set_wait_fault): poll limit and withheld signal for the next launches of this thread.
 thread_local unsigned int g_test_wait_limit = 0;       // 0: the kernels' own limits
 thread_local int g_test_withhold = 0;
+thread_local int g_gram_loader = 0;    // tensor-memory Gram kernel of the latest call: 0 not used, 1 16-byte copies, 2 tensor copies
 
 constexpr int kMaxDevices = 64;
 
@@ -174,6 +175,70 @@ size_t pairwise_extra_bytes(int K) {
     return a > b ? a : b;
 }
 
+// The driver's tensor-map encoder, fetched once through the runtime (the library does not link the driver).
+using TensorMapEncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn tensor_map_encoder() {
+    static std::atomic<void *> fn{nullptr};
+    static std::atomic<int> tried{0};
+    if (!tried.load(std::memory_order_acquire)) {
+        std::lock_guard<std::mutex> lock(g_plan_mutex);
+        if (!tried.load(std::memory_order_relaxed)) {
+            void *p = nullptr;
+            cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+                q != cudaDriverEntryPointSuccess)
+                p = nullptr;
+            cudaGetLastError();
+            fn.store(p, std::memory_order_relaxed);
+            tried.store(1, std::memory_order_release);
+        }
+    }
+    return reinterpret_cast<TensorMapEncodeFn>(fn.load(std::memory_order_relaxed));
+}
+
+#ifndef GAF_TC_L2_PROMOTION
+#define GAF_TC_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_128B
+#endif
+
+// The K bfloat16 gradients as one tensor for tensor copies: possible when they are rows of one matrix (equal,
+// positive distances between their addresses, multiples of 128 bytes), at least one whole 64-element chunk long,
+// and every element coordinate a tile can ask for fits 32 bits.  `tile_map` sees {64 elements, D / 64 chunks, K
+// gradients} and copies boxes of {64, R, Kp}: R consecutive chunks (R x 128 contiguous bytes) of each gradient;
+// `row_map` sees {D elements, K gradients} and copies one 64-element row at a time (the ragged last chunk).  Both
+// with the 128-byte swizzle; what lies outside reads as zero.
+bool stacked_tensor_maps(const void *const *grads, int K, int Kp, int64_t D, int64_t tile_elems, CUtensorMap *tile_map,
+                         CUtensorMap *row_map) {
+    if (K < 2 || Kp < 32 || D < 64 || !aligned16(grads[0])) return false;
+    const intptr_t base = reinterpret_cast<intptr_t>(grads[0]);
+    const intptr_t stride = reinterpret_cast<intptr_t>(grads[1]) - base;
+    if (stride < intptr_t(D) * 2 || (stride & 127) != 0 || stride >= (intptr_t(1) << 40)) return false;
+    for (int i = 2; i < K; ++i)
+        if (reinterpret_cast<intptr_t>(grads[i]) != base + intptr_t(i) * stride) return false;
+    if (D + tile_elems >= (int64_t(1) << 31)) return false;
+    const TensorMapEncodeFn encode = tensor_map_encoder();
+    if (!encode) return false;
+    void *const origin = const_cast<void *>(grads[0]);
+    {
+        const cuuint64_t dims[3] = {64u, cuuint64_t(D / 64), cuuint64_t(K)};
+        const cuuint64_t strides[2] = {128u, cuuint64_t(stride)};
+        const cuuint32_t box[3] = {64u, cuuint32_t(128 / Kp), cuuint32_t(Kp)};
+        const cuuint32_t elem_strides[3] = {1u, 1u, 1u};
+        if (encode(tile_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, origin, dims, strides, box, elem_strides,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, GAF_TC_L2_PROMOTION,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    const cuuint64_t dims[2] = {cuuint64_t(D), cuuint64_t(K)};
+    const cuuint64_t strides[1] = {cuuint64_t(stride)};
+    const cuuint32_t box[2] = {64u, 1u};
+    const cuuint32_t elem_strides[2] = {1u, 1u};
+    return encode(row_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, origin, dims, strides, box, elem_strides,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, GAF_TC_L2_PROMOTION,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tiled Gram matrix of K gradients (by original index) into the workspace; optional
 // distance matrix.  Two launches.
 int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, float *dist_out,
@@ -222,10 +287,18 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         if (slices < 1) slices = 1;
         a.slices = int(slices);
         const int dyn = kTcStages * kTcStageBytes + 1024;
-        auto kernel = t.Kp == 64 ? gram_tc_kernel<true> : gram_tc_kernel<false>;
+        // gradients that are rows of one matrix are fetched by tensor copies, any others by 16-byte copies
+        alignas(64) CUtensorMap tmap, tmap_row;
+        std::memset(&tmap, 0, sizeof tmap);
+        std::memset(&tmap_row, 0, sizeof tmap_row);
+        const bool tma = stacked_tensor_maps(grads, K, t.Kp, D, unit, &tmap, &tmap_row);
+        g_gram_loader = tma ? 2 : 1;
+        void (*kernel)(GramTcArgs, CUtensorMap, CUtensorMap) =
+            t.Kp == 64 ? (tma ? gram_tc_kernel<true, true> : gram_tc_kernel<true, false>)
+                       : (tma ? gram_tc_kernel<false, true> : gram_tc_kernel<false, false>);
         {
-            static PerDevice<DynSmemPlan> table[2];
-            const int w = t.Kp == 64 ? 1 : 0;
+            static PerDevice<DynSmemPlan> table[4];
+            const int w = (t.Kp == 64 ? 1 : 0) + (tma ? 2 : 0);
             if (int rc = plan_once(table[w].plan[di.dev], table[w].ready[di.dev], [&](DynSmemPlan &pl) {
                     pl.dyn = dyn;
                     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) == cudaSuccess
@@ -235,7 +308,7 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         }
         t.spin_limit = g_test_wait_limit ? g_test_wait_limit : kTcSpinLimit;
         t.test_extra_arrival = g_test_withhold;
-        kernel<<<a.slices, t.Kp == 64 ? kTcThreadsWide : kTcThreads, dyn, st>>>(t);
+        kernel<<<a.slices, tc_threads(t.Kp == 64, tma), dyn, st>>>(t, tmap, tmap_row);
         ++g_launches;
     } else {
         // CUDA cores, every gradient read once: one warp per tile pair, panels of D through shared memory
@@ -623,6 +696,7 @@ const char *gaf_error_string(int code) {
 
 int gaf_last_launch_count(void) { return g_launches; }
 int gaf_last_schedule(void) { return g_schedule; }
+int gaf_last_gram_loader(void) { return g_gram_loader; }
 
 int gaf_test_set_wait_fault(unsigned int wait_limit, int withhold) {
     g_test_wait_limit = wait_limit;
@@ -639,7 +713,7 @@ int gaf_workspace_bytes(int K, int64_t D, int dtype, size_t *bytes_out) {
 
 int gaf_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_stream) {
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (cudaMemsetAsync(workspace, 0, kControlBytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return GAF_ERR_CUDA;
     return GAF_OK;
@@ -647,7 +721,7 @@ int gaf_workspace_init(void *workspace, size_t workspace_bytes, void *cuda_strea
 
 int gaf_cosdist(const void *x, const void *y, int64_t D, int dtype, float *dist_out,
                 double *stats_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (((!x || !y) && D > 0) || !dist_out || D < 0) return GAF_ERR_ARG;
     if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
     if (!aligned16(x) || !aligned16(y)) return GAF_ERR_ALIGN;
@@ -671,7 +745,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
                           const int32_t *order, float *macro_out, uint8_t *mask_out,
                           float *dist_out, int32_t *count_out, void *workspace,
                           size_t workspace_bytes, int schedule, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if ((!macro_out && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
     if (schedule < GAF_SCHED_AUTO || schedule > GAF_SCHED_GRAM_FUSED) return GAF_ERR_ARG;
@@ -714,7 +788,7 @@ int gaf_filter_accumulate(const void *const *grads, int K, int64_t D, int dtype,
         if (rc != GAF_OK && library_choice && schedule == GAF_SCHED_GRAM_FUSED) {
             // the launch was refused (for example no CTA of this kernel fits an SM of this device): the
             // library's own choice falls back to the two-launch form, an explicit request does not
-            g_launches = 0;
+            g_launches = 0; g_gram_loader = 0;
             g_schedule = GAF_SCHED_GRAM;
             rc = run(false);
         }
@@ -731,7 +805,7 @@ int gaf_filter_accumulate_repeat(int repeats, int n_sets, const void *const *gra
                                  int dtype, double tau, const int32_t *order, float *macro_out,
                                  uint8_t *mask_out, float *dist_out, int32_t *count_out, void *workspace,
                                  size_t workspace_bytes, int schedule, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (repeats < 0 || n_sets < 1 || !grads || K < 1 || K > GAF_MAX_K) return GAF_ERR_ARG;
     int launches = 0;
     for (int r = 0; r < repeats; ++r) {
@@ -749,7 +823,7 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
                                    float *macro_out, uint8_t *mask_out, float *dist_out,
                                    int32_t *count_out, int32_t *seed_out, void *workspace,
                                    size_t workspace_bytes, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if ((!macro_out && D > 0) || !mask_out || !count_out || !seed_out) return GAF_ERR_ARG;
     if (tau != tau) return GAF_ERR_ARG;
@@ -784,7 +858,7 @@ int gaf_filter_accumulate_any_seed(const void *const *grads, int K, int64_t D, i
     const bool one_launch = auto_one_launch(K, D, dtype);
     int rc = run(one_launch);
     if (rc != GAF_OK && one_launch) {       // launch refused: two launches
-        g_launches = 0;
+        g_launches = 0; g_gram_loader = 0;
         rc = run(false);
     }
     return rc;
@@ -794,7 +868,7 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
                                    const int32_t *order, int S, const int64_t *offsets, float *macro_out,
                                    uint8_t *mask_out, float *dist_out, int32_t *count_out, void *workspace,
                                    size_t workspace_bytes, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if (K > kGsMaxK) return GAF_ERR_UNSUPPORTED;
     if ((!macro_out && D > 0) || !mask_out || !count_out || !offsets || tau != tau) return GAF_ERR_ARG;
@@ -865,7 +939,7 @@ int gaf_filter_accumulate_bucketed(const void *const *grads, int K, int64_t D, i
 
 int gaf_stream_begin(const void *seed, int64_t D, int dtype, float *acc, void *workspace,
                      size_t workspace_bytes, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if ((!seed && D > 0) || (!acc && D > 0) || D < 0) return GAF_ERR_ARG;
     if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
     if (!aligned16(seed) || !aligned16(acc)) return GAF_ERR_ALIGN;
@@ -890,7 +964,7 @@ int gaf_stream_begin(const void *seed, int64_t D, int dtype, float *acc, void *w
 
 int gaf_stream_push(const void *g, int t, int64_t D, int dtype, double tau, float *acc, void *workspace,
                     size_t workspace_bytes, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if ((!g && D > 0) || (!acc && D > 0) || D < 0 || t < 1 || t >= GAF_MAX_K || tau != tau) return GAF_ERR_ARG;
     if (dtype != GAF_F32 && dtype != GAF_BF16) return GAF_ERR_ARG;
     if (!aligned16(g) || !aligned16(acc)) return GAF_ERR_ALIGN;
@@ -926,7 +1000,7 @@ int gaf_stream_push(const void *g, int t, int64_t D, int dtype, double tau, floa
 
 int gaf_stream_end(int K, int64_t D, float *acc, uint8_t *mask_out, float *dist_out, int32_t *count_out,
                    void *workspace, size_t workspace_bytes, void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (K < 1 || K > GAF_MAX_K || D < 0 || (!acc && D > 0) || !mask_out || !count_out) return GAF_ERR_ARG;
     if (!aligned16(acc)) return GAF_ERR_ALIGN;
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset)) return rc;
@@ -953,7 +1027,7 @@ int gaf_filter_accumulate_host(const void *const *grads_host, int K, int64_t D, 
                                int32_t *count_out_host, void *staging, size_t staging_bytes,
                                void *workspace, size_t workspace_bytes, int schedule,
                                void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     size_t need = 0;
     if (int rc = gaf_host_staging_bytes(K, D, dtype, &need)) return rc;
     if (!grads_host || (!macro_out_host && D > 0) || !mask_out_host || !count_out_host) return GAF_ERR_ARG;
@@ -990,7 +1064,7 @@ int gaf_filter_accumulate_host(const void *const *grads_host, int K, int64_t D, 
 int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype, float *dist_out,
                          double *gram_out, void *workspace, size_t workspace_bytes,
                          void *cuda_stream) {
-    g_launches = 0;
+    g_launches = 0; g_gram_loader = 0;
     if (int rc = check_grads(grads, K, D, dtype)) return rc;
     if (!dist_out) return GAF_ERR_ARG;
     if (int rc = check_workspace(workspace, workspace_bytes, kExtraOffset + pairwise_extra_bytes(K)))

@@ -8,16 +8,31 @@
 //
 // Shape of one MMA: the K gradients are too few to fill the 128 rows of a tile, so R =
 // 128 / Kp different 64-element chunks of the D axis are stacked in the rows (Kp = K
-// rounded up to 8, 16, 32 or 64): row c*Kp + i holds 64 consecutive elements of gradient i
-// taken from chunk c.  The same shared-memory tile serves as both operands (A = B, both
-// K-major, 128-byte swizzle), so D = A A^T is 128 x 128 and its R diagonal Kp x Kp blocks
-// are R partial Gram matrices; the off-diagonal blocks mix different chunks and are
-// ignored.
+// rounded up to 8, 16, 32 or 64).  The same shared-memory tile serves as both operands (A = B,
+// both K-major, 128-byte swizzle), so D = A A^T is 128 x 128; the entries whose row and column
+// hold the same chunk are R partial Gram matrices, the others mix different chunks and are
+// ignored.  Two row orders, one per way of filling the tiles:
+//   chunk-major     row c Kp + i = chunk c of gradient i: the partial Gram matrices are the R
+//                   diagonal Kp x Kp blocks (16-byte-copy loaders);
+//   gradient-major  row i R + c: R consecutive chunks of a gradient sit in consecutive rows, which
+//                   is what one tensor copy of a {64 elements, R chunks, Kp gradients} box writes
+//                   and lets it fetch R x 128 contiguous bytes per gradient; the partial Gram
+//                   matrix of chunk c is then the entries (i R + c, j R + c), picked out of all
+//                   128 columns by the epilogue.
 //
 // Pipeline per CTA (one CTA per SM; tiles of the D axis are dealt round-robin to the CTAs):
-//   warps 4-11 loaders: 16-byte cp.async copies global -> swizzled shared memory, a ring of
-//              kTcStages tiles of 64 KB, each copy batch arriving on the tile's mbarrier by itself;
-//   warp 12    one thread issues the MMAs (16 per tile, K = 16 each) into one of two
+//   loaders    a ring of kTcStages tiles of 64 KB in swizzled shared memory, filled in one of two ways.
+//              TMA form (the gradients are rows of one matrix: equal distances, multiples of 128
+//              bytes, between their addresses): one thread of warp 4 issues one tensor copy
+//              (cp.async.bulk.tensor) per 16 KB block, completing on the tile's mbarrier by byte
+//              count; chunks past the end and gradients past K arrive as zeros, and the one block
+//              that holds a ragged last chunk is fetched row by row through a second, element-
+//              granular map.  Measured at 32 gradients: 0.120 ms against 0.134 ms with the 16-byte
+//              copies at D = 11.2 M (6.0 TB/s), 1.27 against 1.41 ms at D = 124 M; a box of one chunk of
+//              every gradient (128 contiguous bytes per gradient) ran at 3.7 TB/s only.
+//              Otherwise warps 4-11 issue 16-byte cp.async copies, each thread's batch arriving on
+//              the mbarrier by itself;
+//   MMA warp   one thread issues the MMAs (16 per tile, K = 16 each) into one of two
 //              128-column accumulator buffers in tensor memory and commits to mbarriers;
 //   warps 0-3  epilogue: every kTcDrain tiles read the finished buffer with tcgen05.ld and
 //              add it to binary64 registers (short binary32 accumulation chains only).
@@ -29,6 +44,8 @@
 // Gram matrix in the [tile pair][slice][64] layout of the CUDA-core version, so the same
 // finishing kernel totals the slices.  Every wait is bounded.
 #pragma once
+
+#include <cuda.h>        // CUtensorMap (the type only: the encoder is fetched from the driver at run time)
 
 #include "gaf_device.cuh"
 
@@ -45,9 +62,6 @@ namespace gaf {
 #endif
 constexpr int kTcLoaderWarps = GAF_TC_LOADER_WARPS;
 constexpr int kTcLoaders = kTcLoaderWarps * 32;
-constexpr int kTcMmaWarp = 4 + kTcLoaderWarps;  // warps 0-3 epilogue, then the loaders, then the MMA issuer
-constexpr int kTcThreads = (kTcMmaWarp + 1) * 32;
-constexpr int kTcThreadsWide = kTcThreads + 128;  // 33..64 gradients: four more epilogue warps after the MMA warp
 constexpr int kTcStages = GAF_TC_STAGES;
 constexpr int kTcSub = GAF_TC_SUB;              // 128-row x 128-byte swizzle blocks per tile (one handshake per tile)
 constexpr int kTcBlockBytes = 128 * 128;        // one such block: 128 rows x 128 bytes
@@ -128,6 +142,28 @@ __device__ __forceinline__ void tc_cp_async16_zfill(uint32_t dst_smem, const voi
 __device__ __forceinline__ void tc_cp_async_arrive(uint64_t *bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(tc_smem_u32(bar)) : "memory");
 }
+// One arrival that also announces `bytes` of asynchronous copies to come (the phase completes when both the
+// arrivals and the bytes are in).
+__device__ __forceinline__ void tc_mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tc_smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Tensor copy of one box of a two-dimensional tensor map into (swizzled) shared memory; x is the element
+// coordinate along D (a multiple of 64 here, so the copy starts on a 128-byte boundary), y the first row.
+__device__ __forceinline__ void tc_tma_load_2d(uint32_t dst_smem, const CUtensorMap *map, int32_t x, int32_t y,
+                                               uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(tc_smem_u32(bar))
+        : "memory");
+}
+// The same for a box of a three-dimensional map ({element, chunk, gradient}; x = 0 here).
+__device__ __forceinline__ void tc_tma_load_3d(uint32_t dst_smem, const CUtensorMap *map, int32_t x, int32_t y, int32_t z,
+                                               uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(tc_smem_u32(bar))
+        : "memory");
+}
 __device__ __forceinline__ void tc_cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -187,9 +223,21 @@ struct GramTcShared {
 // WIDE: Kp = 64.  A row's diagonal block is then 64 columns wide, twice what one epilogue thread can
 // carry in binary64 registers, so a second set of four epilogue warps (after the MMA warp; a warp reads
 // the tensor-memory lanes 32 (warp mod 4) .. + 31) takes the upper 32 columns of each block.
-template <bool WIDE>
-__global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc_kernel(const __grid_constant__ GramTcArgs a) {
-    constexpr int kThreads = WIDE ? kTcThreadsWide : kTcThreads;
+//
+// TMA: the tiles are filled by tensor copies, gradient-major rows (Kp is 32 or 64 then): `tmap` has the
+// dimensions {64, D / 64, K} of bfloat16 and the box {64, R, Kp}, `tmap_row` the dimensions {D, K} and the box
+// {64, 1}; both with the 128-byte swizzle and zero fill outside.  Otherwise neither map is touched.
+// Threads of a launch: four epilogue warps, the loader warps (one with tensor copies), the MMA warp, and four
+// more epilogue warps for 33..64 gradients.
+__host__ __device__ constexpr int tc_mma_warp(bool tma) { return 4 + (tma ? 1 : kTcLoaderWarps); }
+__host__ __device__ constexpr int tc_threads(bool wide, bool tma) { return (tc_mma_warp(tma) + 1) * 32 + (wide ? 128 : 0); }
+
+template <bool WIDE, bool TMA>
+__global__ void __launch_bounds__(tc_threads(WIDE, TMA), 1)
+gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUtensorMap tmap,
+               const __grid_constant__ CUtensorMap tmap_row) {
+    constexpr int kThreads = tc_threads(WIDE, TMA);
+    constexpr int kMmaWarp = tc_mma_warp(TMA);
     extern __shared__ unsigned char tc_dyn_smem[];
     __shared__ GramTcShared sh;
 
@@ -211,8 +259,8 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
-            // every loader thread arrives
-            tc_mbar_init(&sh.full[s], kTcLoaders + ((s == 0 && a.test_extra_arrival) ? 1 : 0));
+            // every loader thread arrives (TMA form: the issuing thread, plus the tile's bytes)
+            tc_mbar_init(&sh.full[s], (TMA ? 1 : kTcLoaders) + ((s == 0 && a.test_extra_arrival) ? 1 : 0));
             tc_mbar_init(&sh.empty[s], 1);               // one commit
         }
         for (int b = 0; b < 2; ++b) {
@@ -224,15 +272,15 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         if (blockIdx.x == 0) a.ctl->status = 0;          // first kernel of the operation
     }
-    // rows of absent gradients (K < Kp) stay zero for the whole kernel
-    if (K < Kp) {
+    // rows of absent gradients (K < Kp) stay zero for the whole kernel (the tensor copies write them as zeros)
+    if (!TMA && K < Kp) {
         for (int idx = threadIdx.x; idx < kTcStages * kTcSub * 128 * 8; idx += kThreads) {
             const int row = (idx >> 3) & 127;
             if ((row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
         }
         tc_fence_async_smem();
     }
-    if (warp == kTcMmaWarp) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&sh.tmem_base)),
                      "r"(kTcTmemCols)
                      : "memory");
@@ -245,14 +293,57 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
 
     // epilogue warps: which 32 rows (tensor-memory lanes) and which 32 columns of them this warp reads --
     // the columns that hold the rows' diagonal block(s): the 32 on the diagonal, or one half of the 64
+    // (gradient-major rows: the first of all 128 columns, or of the half that holds this warp set's 32 gradients)
     const int epi_q = warp & 3;
-    const int epi_col0 = WIDE ? (epi_q >> 1) * 64 + (warp > kTcMmaWarp ? 32 : 0) : epi_q * 32;
+    const int epi_col0 = TMA ? ((WIDE && warp > kMmaWarp) ? 64 : 0)
+                             : (WIDE ? (epi_q >> 1) * 64 + (warp > kMmaWarp ? 32 : 0) : epi_q * 32);
     double gsum[32];                                     // epilogue: this row's 32 loaded columns
 #pragma unroll
     for (int j = 0; j < 32; ++j) gsum[j] = 0.0;
 
-    if (warp >= 4 && warp < kTcMmaWarp) {
-        // ------------------------------------------------------ loaders --------
+    if (TMA && warp >= 4 && warp < kMmaWarp) {
+        // ------------------------------------------------------ loader (tensor copies) ----
+        // (one warp; lane 0 does the handshakes and the block copies, all lanes share the row copies)
+        {
+            const int64_t full_chunks = a.D / 64;            // what the chunk-granular map covers
+            const bool ragged = (a.D % 64) != 0;
+            int issued = 0;
+            for (int it = 0; it < n_tiles; ++it) {
+                const int s = it % kTcStages;
+                if (it >= kTcStages &&
+                    !tc_mbar_wait_warp(&sh.empty[s], (uint32_t)((it / kTcStages - 1) & 1), &sh.abort_flag, a.spin_limit))
+                    break;
+                const int64_t elem0 = (blockIdx.x + it * G) * unit;   // first element of the tile, per gradient
+                const uint32_t tile = tiles_u32 + (uint32_t)s * kTcStageBytes;
+                if (lane == 0) tc_mbar_arrive_expect_tx(&sh.full[s], (uint32_t)kTcStageBytes);
+                __syncwarp();
+                for (int b = 0; b < kTcSub; ++b) {
+                    // block b: chunks chunk0 .. chunk0 + R - 1 of every gradient, row i R + c
+                    const int64_t chunk0 = elem0 / 64 + (int64_t)b * R;
+                    const uint32_t block = tile + (uint32_t)b * kTcBlockBytes;
+                    if (!(ragged && chunk0 <= full_chunks && full_chunks < chunk0 + R)) {
+                        if (lane == 0) tc_tma_load_3d(block, &tmap, 0, (int32_t)chunk0, 0, &sh.full[s]);
+                    } else {
+                        // the one block of the whole vector that holds the partial last chunk: row by row through
+                        // the element-granular map, which fills what lies past D (and past K) with zeros; the
+                        // lanes issue four rows each (one thread issuing all 128 took 5 us)
+                        for (int row = lane; row < 128; row += 32)
+                            tc_tma_load_2d(block + (uint32_t)row * 128u, &tmap_row,
+                                           (int32_t)((chunk0 + row % R) * 64), row / R, &sh.full[s]);
+                    }
+                }
+                issued = it + 1;
+            }
+            // The last copies must have landed before the CTA leaves its shared memory to the next one, also when
+            // a wait gave up somewhere and nobody consumes them (bounded like every wait; ignores the abort flag).
+            if (lane == 0)
+                for (int it = issued > kTcStages ? issued - kTcStages : 0; it < issued; ++it)
+                    for (unsigned int spin = 0; spin < a.spin_limit; ++spin)
+                        if (tc_mbar_try(&sh.full[it % kTcStages], (uint32_t)((it / kTcStages) & 1), 2000u)) break;
+        }
+        __syncwarp();
+    } else if (warp >= 4 && warp < kMmaWarp) {
+        // ------------------------------------------------------ loaders (16-byte copies) ----
         const int tl = threadIdx.x - 128;                // 0..kTcLoaders-1
         const int run = kTcSub * R * 8;                  // 16-byte pieces of one gradient in a tile (contiguous)
         const int pieces = K * run;                      // 16-byte pieces per tile
@@ -305,7 +396,7 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
             tc_cp_async_arrive(&sh.full[s]);
         }
         tc_cp_async_wait_all();
-    } else if (warp == kTcMmaWarp) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------------ MMA issuer -----
         if (lane == 0) {
             for (int it = 0; it < n_tiles; ++it) {
@@ -317,9 +408,9 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
                     if (!tc_mbar_wait(&sh.acc_empty[buf], (uint32_t)((blk / 2 - 1) & 1), &sh.abort_flag, a.spin_limit)) break;
                 }
                 if (!tc_mbar_wait(&sh.full[s], (uint32_t)((it / kTcStages) & 1), &sh.abort_flag, a.spin_limit)) break;
-                // the tile was written by cp.async (generic proxy) and is read by the MMA through the
-                // asynchronous proxy: order the two before the first MMA of the tile
-                tc_fence_async_smem();
+                // a tile written by cp.async (generic proxy) is read by the MMA through the asynchronous
+                // proxy: order the two before the first MMA of the tile (tensor copies are of that proxy already)
+                if (!TMA) tc_fence_async_smem();
                 tc_fence_after_sync();
 #pragma unroll
                 for (int b = 0; b < kTcSub; ++b) {
@@ -350,11 +441,39 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
             if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag, a.spin_limit)) break;
             tc_fence_after_sync();
             uint32_t r[32];
-            tc_tmem_ld32(tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128 + epi_col0), r);
-            tc_fence_before_sync();
-            tc_mbar_arrive(&sh.acc_empty[buf]);
+            const uint32_t taddr = tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128 + epi_col0);
+            if constexpr (!TMA) {
+                tc_tmem_ld32(taddr, r);
+                tc_fence_before_sync();
+                tc_mbar_arrive(&sh.acc_empty[buf]);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) gsum[j] += (double)__uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) gsum[j] += (double)__uint_as_float(r[j]);
+            } else {
+                // this row holds chunk c of its gradient: its Gram entries are the columns j R + c
+                constexpr int RR = WIDE ? 2 : 4;             // R
+                constexpr int kPer = 32 / RR;                // gradients per 32 loaded columns
+                const int c = lane & (RR - 1);
+#pragma unroll
+                for (int t = 0; t < RR; ++t) {
+                    tc_tmem_ld32(taddr + (uint32_t)(32 * t), r);
+                    if (t == RR - 1) {
+                        tc_fence_before_sync();
+                        tc_mbar_arrive(&sh.acc_empty[buf]);
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < kPer; ++jj) {
+                        uint32_t v;
+                        if constexpr (WIDE) {
+                            v = c ? r[2 * jj + 1] : r[2 * jj];
+                        } else {
+                            const uint32_t lo = (c & 1) ? r[4 * jj + 1] : r[4 * jj];
+                            const uint32_t hi = (c & 1) ? r[4 * jj + 3] : r[4 * jj + 2];
+                            v = (c & 2) ? hi : lo;
+                        }
+                        gsum[t * kPer + jj] += (double)__uint_as_float(v);
+                    }
+                }
+            }
         }
     }
 
@@ -362,7 +481,7 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == kTcMmaWarp) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols) : "memory");
     }
     if (sh.abort_flag) {
@@ -374,14 +493,21 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) gram_tc
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles <= 64 KB)
     double *red = reinterpret_cast<double *>(tiles);
-    if (warp < 4 || warp > kTcMmaWarp) {
+    if (warp < 4 || warp > kMmaWarp) {
         const int row = epi_q * 32 + lane;               // row of the 128 x 128 result
-        const int c = row / Kp, i = row % Kp;
-        const int off = c * Kp - epi_col0;               // where this chunk's block starts in the loaded columns
+        if constexpr (TMA) {
+            const int i = row / R, c = row % R;
+            const int j0 = (WIDE && warp > kMmaWarp) ? 32 : 0;   // first gradient of this warp set's columns
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const int jj = j - off;
-            if (jj >= 0 && jj < Kp) red[((size_t)c * Kp + i) * Kp + jj] = gsum[j];
+            for (int j = 0; j < 32; ++j) red[((size_t)c * Kp + i) * Kp + j0 + j] = gsum[j];
+        } else {
+            const int c = row / Kp, i = row % Kp;
+            const int off = c * Kp - epi_col0;           // where this chunk's block starts in the loaded columns
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int jj = j - off;
+                if (jj >= 0 && jj < Kp) red[((size_t)c * Kp + i) * Kp + jj] = gsum[j];
+            }
         }
     }
     __syncthreads();

@@ -92,13 +92,19 @@ def as_numpy_bits(t: torch.Tensor) -> np.ndarray:
 
 
 def _draw(K: int, D: int, dtype: str, rho: Sequence[float], seed: int,
-          device: str, sigma, chunk: int = 1 << 24) -> List[torch.Tensor]:
+          device: str, sigma, chunk: int = 1 << 24, stacked: bool = False) -> List[torch.Tensor]:
     """Draw K micro-gradients of D elements.  ``sigma`` is a float or a
-    per-element float32 tensor on ``device``."""
+    per-element float32 tensor on ``device``.  ``stacked``: the gradients are the
+    rows of one matrix whose row stride is D rounded up to 128 elements (what an
+    all-gather of padded flat gradients leaves); the values are the same either way."""
     tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
-    grads = [torch.empty(D, dtype=tdtype, device=device) for _ in range(K)]
+    if stacked:
+        matrix = torch.zeros(K, (D + 127) // 128 * 128, dtype=tdtype, device=device)
+        grads = [matrix[i, :D] for i in range(K)]
+    else:
+        grads = [torch.empty(D, dtype=tdtype, device=device) for _ in range(K)]
     alpha = [math.copysign(math.sqrt(abs(r)), r) for r in rho]
     beta = [math.sqrt(1.0 - abs(r)) for r in rho]
     for lo in range(0, D, chunk):
@@ -117,18 +123,18 @@ def _clip_rho(r: Sequence[float]) -> List[float]:
 
 def mixture(K: int, D: int, dtype: str, rho: Sequence[float], seed: int,
             device: str = "cpu", sigma=1e-3, taus: Sequence[float] = (0.97,),
-            name: str = "custom") -> Workload:
+            name: str = "custom", stacked: bool = False) -> Workload:
     """A workload with explicit rho values (used by the tests for small and
     ragged shapes)."""
     rho = _clip_rho(rho)
     assert len(rho) == K
     w = Workload(name, K, D, dtype, [float(t) for t in taus], rho, seed)
-    w.grads = _draw(K, D, dtype, rho, seed, device, sigma)
+    w.grads = _draw(K, D, dtype, rho, seed, device, sigma, stacked=stacked)
     return w
 
 
 def config(n: int, device: str = "cpu", D: Optional[int] = None,
-           K: Optional[int] = None, seed: Optional[int] = None) -> Workload:
+           K: Optional[int] = None, seed: Optional[int] = None, stacked: bool = False) -> Workload:
     """Named configuration ``n`` (1..5).  ``D``/``K`` override the size for
     scaled-down copies of the same recipe (the tensor layout of configuration 2
     is kept only at its native D); ``seed`` draws another instance of it."""
@@ -170,5 +176,5 @@ def config(n: int, device: str = "cpu", D: Optional[int] = None,
         sigma = torch.repeat_interleave(torch.from_numpy(per_tensor),
                                         torch.tensor(sizes)).to(device)
     w = Workload(f"config{n}", K_, D_, dtype, taus, rho, seed)
-    w.grads = _draw(K_, D_, dtype, rho, seed, device, sigma)
+    w.grads = _draw(K_, D_, dtype, rho, seed, device, sigma, stacked=stacked)
     return w

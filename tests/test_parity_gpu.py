@@ -22,11 +22,23 @@ def ws():
     return gaf.new_workspace(gaf.binding.GAF_MAX_K, 1 << 20, gaf.GAF_F32)
 
 
-def _mix(K, D, dtype, seed, rho=None, sigma=1e-3):
+def _mix(K, D, dtype, seed, rho=None, sigma=1e-3, stacked=False):
     rng = np.random.RandomState(seed)
     if rho is None:
         rho = rng.uniform(-0.4, 0.9, size=K)
-    return workloads.mixture(K, D, dtype, list(rho), seed, device="cuda", sigma=sigma)
+    return workloads.mixture(K, D, dtype, list(rho), seed, device="cuda", sigma=sigma, stacked=stacked)
+
+
+def _scattered(grads):
+    """The same gradients at unequal distances from one another: rows of a wider matrix, two of them swapped."""
+    K, D = len(grads), grads[0].numel()
+    matrix = torch.empty(K + 1, (D + 127) // 128 * 128 + 128, dtype=grads[0].dtype, device=grads[0].device)
+    rows = list(range(K))
+    rows[1], rows[K - 1] = K, 1
+    out = [matrix[r, :D] for r in rows]
+    for o, g in zip(out, grads):
+        o.copy_(g)
+    return out
 
 
 # ------------------------------------------------------------------ Eq. 4 ----
@@ -395,23 +407,30 @@ def test_bounded_waits_run_out_and_the_workspace_recovers(ws):
         # one-launch Gram-first schedule: the waiting CTAs are never shown the full arrival counter
         (_mix(4, 600_011, "f32", seed=11, rho=[0.8, 0.6, -0.2, 0.7]), gaf.GAF_SCHED_GRAM_FUSED),
         (_mix(8, 300_007, "bf16", seed=12), gaf.GAF_SCHED_GRAM_FUSED),
-        # tcgen05 Gram pipeline (17..64 bfloat16 gradients): the first tile's barrier never completes
-        (_mix(17, 300_007, "bf16", seed=13), gaf.GAF_SCHED_GRAM),
-        (_mix(40, 100_003, "bf16", seed=14), gaf.GAF_SCHED_GRAM),
+        # tcgen05 Gram pipeline (17..64 bfloat16 gradients): the first tile's barrier never completes --
+        # with the 16-byte-copy loaders (gradients anywhere) ...
+        (_scattered(_mix(17, 300_007, "bf16", seed=13).grads), gaf.GAF_SCHED_GRAM, 1),
+        (_scattered(_mix(40, 100_003, "bf16", seed=14).grads), gaf.GAF_SCHED_GRAM, 1),
+        # ... and with the tensor-copy loader (gradients that are rows of one matrix), ragged and whole last chunk
+        (_mix(17, 300_007, "bf16", seed=13, stacked=True), gaf.GAF_SCHED_GRAM, 2),
+        (_mix(40, 64 * 1500, "bf16", seed=14, stacked=True), gaf.GAF_SCHED_GRAM, 2),
     ]
-    for w, schedule in cases:
+    cases = [(c[0] if isinstance(c[0], list) else c[0].grads, c[1], c[2] if len(c) > 2 else 0) for c in cases]
+    for grads, schedule, loader in cases:
         try:
             gaf.gaf_test_set_wait_fault(1000, True)
-            gaf.gaf_filter_accumulate(w.grads, 0.97, ws, schedule=schedule)
+            gaf.gaf_filter_accumulate(grads, 0.97, ws, schedule=schedule)
             status = gaf.gaf_read_status(ws)
         finally:
             gaf.gaf_test_set_wait_fault(0, False)
         assert status & gaf.GAF_STATUS_TIMEOUT, (schedule, status)
-        check_filter(w.grads, 0.97, ws, schedule=schedule)
+        assert gaf.gaf_last_gram_loader() == loader
+        check_filter(grads, 0.97, ws, schedule=schedule)
     # a short limit alone, with the signal given, must not time out
     try:
         gaf.gaf_test_set_wait_fault(1 << 20, False)
-        check_filter(cases[0][0].grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED)
+        check_filter(cases[0][0], 0.97, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED)
+        check_filter(cases[-1][0], 0.97, ws, schedule=gaf.GAF_SCHED_GRAM)
     finally:
         gaf.gaf_test_set_wait_fault(0, False)
 
@@ -640,9 +659,40 @@ def test_pairwise_zero_norm_row(ws):
     assert bool((dist[2] == 1.0).all()) and bool((dist[:, 2] == 1.0).all())
 
 
+@pytest.mark.parametrize("K", [17, 32, 33, 64])
+def test_tensor_copy_loader_of_the_tcgen05_gram_kernel(ws, K):
+    """bfloat16 gradients that are rows of one matrix are fetched by tensor copies (gradient-major tile rows, the
+    epilogue picks the Gram entries out of all columns), any other placement by 16-byte copies (chunk-major rows):
+    both against the oracle and against each other, for every kind of end of the vector -- shorter than a chunk
+    (no tensor copies), one whole chunk, a ragged chunk in each position of its block, whole chunks that do not
+    fill the last block or tile, several tiles."""
+    sizes = (40, 64, 65, 64 + 63, 200, 64 * 7, 64 * 8 + 1, 3072 + 192, 3072 + 192 + 17, 70_001, 262_152, 1_000_003)
+    for D in sizes:
+        w = _mix(K, D, "bf16", seed=3 * K + D % 97, stacked=True)
+        check_pairwise(w.grads, ws)
+        assert gaf.gaf_last_gram_loader() == (2 if D >= 64 else 1), D
+        gram_rows = gaf.gaf_pairwise_cosdist(w.grads, ws)[1].clone()
+        elsewhere = _scattered(w.grads)
+        check_pairwise(elsewhere, ws)
+        assert gaf.gaf_last_gram_loader() == 1
+        gram_any = gaf.gaf_pairwise_cosdist(elsewhere, ws)[1]
+        scale = gram_any.diagonal().sqrt()
+        assert float(((gram_rows - gram_any).abs() / scale[:, None] / scale[None, :]).max()) < 2e-6
+    # the filter on top of it, and a row distance that is not a multiple of 128 bytes (16-byte copies then)
+    w = _mix(K, 300_007, "bf16", seed=5 * K, stacked=True)
+    check_filter(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM)
+    assert gaf.gaf_last_gram_loader() == 2
+    tight = torch.stack([g[:300_000] for g in w.grads])                 # rows 600,000 bytes apart
+    check_pairwise(list(tight.unbind(0)), ws)
+    assert gaf.gaf_last_gram_loader() == 1
+
+
 def test_config3_pairwise(ws):
     w = workloads.config(3, device="cuda")
     check_pairwise(w.grads, ws)
+    stacked = workloads.config(3, device="cuda", stacked=True)
+    check_pairwise(stacked.grads, ws)
+    assert gaf.gaf_last_gram_loader() == 2
     dist, _ = gaf.gaf_pairwise_cosdist(w.grads, ws)
     rho = np.array(w.rho)
     want = 1.0 - np.sign(rho)[:, None] * np.sign(rho)[None, :] * np.sqrt(np.abs(np.outer(rho, rho)))
