@@ -102,14 +102,19 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Launch `kernel` as a programmatic dependent of the launch before it on the stream: its blocks may be
 // placed while that grid winds down; the kernel itself waits (griddepcontrol.wait) for that grid.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int threads, cudaStream_t st, const Args &...args) {
+cudaError_t launch_dependent_smem(void (*kernel)(KArgs...), int grid, int threads, size_t dyn_smem, cudaStream_t st,
+                                  const Args &...args) {
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = dyn_smem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int threads, cudaStream_t st, const Args &...args) {
+    return launch_dependent_smem(kernel, grid, threads, 0, st, args...);
 }
 
 // macro_out (D floats) must not overlap any input gradient.
@@ -198,6 +203,8 @@ TensorMapEncodeFn tensor_map_encoder() {
     return reinterpret_cast<TensorMapEncodeFn>(fn.load(std::memory_order_relaxed));
 }
 
+constexpr int kTcTensorCopyMaxWideK = 52;
+
 #ifndef GAF_TC_L2_PROMOTION
 #define GAF_TC_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_128B
 #endif
@@ -211,6 +218,10 @@ TensorMapEncodeFn tensor_map_encoder() {
 bool stacked_tensor_maps(const void *const *grads, int K, int Kp, int64_t D, int64_t tile_elems, CUtensorMap *tile_map,
                          CUtensorMap *row_map) {
     if (K < 2 || Kp < 32 || D < 64 || !aligned16(grads[0])) return false;
+    // 64-row-pair tiles (33..64 gradients) give a box only 256 contiguous bytes per gradient, and the copy engine's
+    // rate falls with the number of separate pieces: measured at D = 11.2 M against the 16-byte copies, 195 / 227 us
+    // against 210 / 238 us at 40 / 52 gradients, but 252 / 272 / 292 against 243 / 250 / 259 us at 56 / 60 / 64.
+    if (Kp == 64 && K > kTcTensorCopyMaxWideK) return false;
     const intptr_t base = reinterpret_cast<intptr_t>(grads[0]);
     const intptr_t stride = reinterpret_cast<intptr_t>(grads[1]) - base;
     if (stride < intptr_t(D) * 2 || (stride & 127) != 0 || stride >= (intptr_t(1) << 40)) return false;
@@ -308,8 +319,12 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         }
         t.spin_limit = g_test_wait_limit ? g_test_wait_limit : kTcSpinLimit;
         t.test_extra_arrival = g_test_withhold;
-        kernel<<<a.slices, tc_threads(t.Kp == 64, tma), dyn, st>>>(t, tmap, tmap_row);
+        // (a programmatic dependent of whatever precedes it on the stream: barriers and tensor memory are set up
+        // while that grid winds down, and the kernel waits for it before it touches global memory)
+        const cudaError_t err = launch_dependent_smem(kernel, a.slices, tc_threads(t.Kp == 64, tma), size_t(dyn), st,
+                                                      t, tmap, tmap_row);
         ++g_launches;
+        if (err != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
     } else {
         // CUDA cores, every gradient read once: one warp per tile pair, panels of D through shared memory
         GramPanelArgs pa{};

@@ -270,7 +270,6 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
         tc_mbar_init(&sh.drained, 1);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (blockIdx.x == 0) a.ctl->status = 0;          // first kernel of the operation
     }
     // rows of absent gradients (K < Kp) stay zero for the whole kernel (the tensor copies write them as zeros)
     if (!TMA && K < Kp) {
@@ -290,6 +289,11 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sh.tmem_base;
+    // Everything above touched only this CTA's shared and tensor memory.  The kernel is launched as a programmatic
+    // dependent of its predecessor on the stream: wait for that grid (its results, and its last reads of the
+    // workspace) before the first access to global memory.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.ctl->status = 0;      // first kernel of the operation
 
     // epilogue warps: which 32 rows (tensor-memory lanes) and which 32 columns of them this warp reads --
     // the columns that hold the rows' diagonal block(s): the 32 on the diagonal, or one half of the 64

@@ -46,6 +46,8 @@ __global__ void __launch_bounds__(64 * kFinishParts) gram_finish_kernel(GramArgs
     // launched as a programmatic dependent of the Gram kernel: wait until that grid has completed
     // and its partial sums are visible (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // a dependent of this launch may be placed now (it waits for this grid before it touches global memory)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     {
         const int per = (a.slices + kFinishParts - 1) / kFinishParts;
         const int lo = chain * per, hi = min(a.slices, lo + per);
