@@ -576,6 +576,35 @@ def measure_cosdist(torch, gaf, workloads, dev, D, steps, nvml, peak, peak_kind)
             "clocks": t["clocks"]}
 
 
+def measure_two_gradients(torch, gaf, workloads, dev, D, steps, nvml, peak, peak_kind):
+    """The filter on two fp32 micro-gradients (the setting of the paper's experiments, Section 4) of configuration 2's
+    recipe at length D, four rotating input sets: a stream of calls that all accept the second gradient (tau = 2), one
+    that all reject it (tau = 0), and one in which the outcome changes with every call."""
+    n_sets = 4 if 3 * 4 * D * 4 < 6e9 else 1
+    sets = [workloads.config(2 if D == FULL_D[2] else 4, device=dev, K=2, D=D, seed=1 + 1000 * i).grads
+            for i in range(n_sets)]
+    ws = gaf.new_workspace(2, D, gaf.GAF_F32, device=dev)
+    macro, mask, dist, count = gaf.gaf_filter_accumulate(sets[0], 2.0, ws)
+    min_b = (2 * 4 + 4) * D
+    out = {"workload": f"gaf_filter_accumulate, K=2, D={D}, f32 inputs ({n_sets} rotating sets)",
+           "op": "gaf_filter_accumulate", "unit": UNIT, "min_bytes_per_call": min_b,
+           "byte_model": "both gradients read once, the output written once when the previous call's outcome repeats: "
+                         "(2 b + 4) D (= the minimum); 20 D when it does not", "peak": peak, "peak_kind": peak_kind}
+    for name, taus in (("all_accepted", (2.0,)), ("all_rejected", (0.0,)), ("alternating", (2.0, 0.0))):
+        def step(i, taus=taus):
+            gaf.gaf_filter_accumulate(sets[i % n_sets], taus[i % len(taus)], ws, macro_out=macro, mask_out=mask,
+                                      dist_out=dist, count_out=count)
+        step(0)
+        launches = gaf.gaf_last_launch_count()
+        t = timed_region(torch, step, steps, 5, nvml)
+        ms = t["ms_per_step"]
+        rate = min_b / (ms * 1e-3) / 1e9
+        out[name] = {"steps": steps, "ms_per_call": ms, "launches_per_call": launches,
+                     "ms_per_call_median_of_event_pairs": statistics.median(t["per_call_ms"]),
+                     "value": 2 * 4 * D / (ms * 1e-3) / 1e9, "min_bytes_frac": rate / peak, "clocks": t["clocks"]}
+    return out
+
+
 def pairwise_entry(m, peak, peak_kind, steps):
     t = m["timing"]
     ms = t["ms_per_step"]
@@ -732,6 +761,14 @@ def run_ours(args):
         for key, D_c, n in (("cosdist_D11.2M", FULL_D[2], 1000), ("cosdist_D124M", FULL_D[4], 200)):
             try:
                 block[key] = measure_cosdist(torch, gaf, workloads, dev, D_c, n, nvml, peak, peak_kind)
+            except Exception as exc:
+                block[key] = {"error": f"{type(exc).__name__}: {exc}"}
+            gc.collect()
+            torch.cuda.empty_cache()
+
+        for key, D_c, n in (("two_gradients_D11.2M", FULL_D[2], 1000), ("two_gradients_D124M", FULL_D[4], 100)):
+            try:
+                block[key] = measure_two_gradients(torch, gaf, workloads, dev, D_c, n, nvml, peak, peak_kind)
             except Exception as exc:
                 block[key] = {"error": f"{type(exc).__name__}: {exc}"}
             gc.collect()

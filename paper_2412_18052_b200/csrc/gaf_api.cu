@@ -614,6 +614,8 @@ int launch_gram_first(const void *const *g, int K, int64_t D, int dtype, double 
 // Whether the library's own choice is the one-launch form of the Gram-first schedule.
 bool auto_one_launch(int K, int64_t D, int dtype) {
     if (!use_small_gram(K, D, dtype)) return false;
+    // two gradients: the one-launch kernel writes their mean during its only pass over them, at any length
+    if (K == 2) return true;
     if (dtype == GAF_F32) return int64_t(K) * 4 * D <= kFusedMaxInputBytesF32;
     return K < 7 || int64_t(K) * 2 * D <= kFusedMaxInputBytesBf16Mma;
 }

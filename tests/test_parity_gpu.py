@@ -619,6 +619,30 @@ def test_auto_schedule_choice(ws):
     assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM and gaf.gaf_last_launch_count() == 2
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_two_gradients_mean_written_in_the_first_pass(ws, dtype):
+    """Two gradients (the setting of the paper's Section 4): the one-launch kernel writes the mean of both while
+    it forms the sums and rewrites the output with the first gradient alone when the second is rejected.  Both
+    outcomes, both orders, ragged lengths, the order-indifferent variant, and bit-identity with the other schedules."""
+    for D in (1, 7, 1001, 300_007, 5_000_003):
+        for rho, tau in (([0.8, 0.7], 0.97), ([0.8, -0.5], 0.97), ([0.3, 0.2], 2.0), ([0.9, 0.9], 0.0)):
+            w = _mix(2, D, dtype, seed=D % 89 + int(10 * tau), rho=rho)
+            for order in (None, [1, 0]):
+                r = check_filter(w.grads, tau, ws, order=order)
+                assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM_FUSED and gaf.gaf_last_launch_count() == 1
+                got = gaf.gaf_filter_accumulate(w.grads, tau, ws, order=order)
+                for schedule in (gaf.GAF_SCHED_GRAM, gaf.GAF_SCHED_STEPWISE):
+                    other = gaf.gaf_filter_accumulate(w.grads, tau, ws, order=order, schedule=schedule)
+                    if torch.equal(other[1], got[1]):                      # (masks may differ on a tie only)
+                        assert torch.equal(other[0], got[0]), (D, rho, tau, order, schedule)
+            check_any_seed(w.grads, tau, ws)
+    # rejected and accepted counts really both occurred above; and at a length beyond the old one-launch limit
+    big = _mix(2, 70_000_003, "f32", seed=5, rho=[0.6, 0.5])
+    check_filter(big.grads, 0.97, ws)
+    assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM_FUSED
+    check_filter(big.grads, 0.0, ws)
+
+
 def test_wide_mma_gram_kernel_shapes_and_long_runs(ws):
     """9..16 bfloat16 gradients (and the first counts of the tcgen05 tile behind them): absent rows feed zeros;
     lengths below one tile, ragged ends, and a length from which the CTAs walk in runs of several trips."""
