@@ -131,17 +131,17 @@ def min_bytes(K, D, b):
 NCU_TRAFFIC = {
     # gram_fused_kernel<float,4> at configuration 2 itself (D = 11,227,812)
     (2, 3): {"sources": ["gaf_fused.cuh", "gaf_gramfilter.cuh", "gaf_device.cuh"],
-             "sha256": "b0251f16d69b2f78f384133653cd9c83ffea9080495cada25e29c219c1acb77f",
-             "steady": {2: 262.7e6 / 11227812, 3: 296.6e6 / 11227812},
-             "flushed": {2: 232.0e6 / 11227812, 3: 259.6e6 / 11227812}},
+             "sha256": "cd6bdf745da44d90ce916c4a701b35e5a478f9ddc0803a520949d2b45e9660ac",
+             "steady": {2: 262.6e6 / 11227812, 3: 296.7e6 / 11227812},
+             "flushed": {2: 230.5e6 / 11227812, 3: 257.9e6 / 11227812}},
     # gram_small_kernel<float,8> + masked_mean_kernel<float>, captured at D = 80,000,000
     (4, 2): {"sources": ["gaf_gramfilter.cuh", "gaf_device.cuh"],
-             "sha256": "605c2ef6d0cc865bb09a5d25d703927c4c13c9bf97bcbaca7df1d0e48b9c36f9",
-             "steady": {4: (2563.4e6 + 1573.8e6) / 80e6, 1: (2563.9e6 + 590.8e6) / 80e6}},
+             "sha256": "707df4a1adb38d5c23a4b0a9334cb7ee98408cb34984959ae16d9bc13231b65d",
+             "steady": {4: (2563.4e6 + 1573.5e6) / 80e6, 1: (2563.9e6 + 591.2e6) / 80e6}},
     # gram_mma_kernel<8> + masked_mean_kernel<bf16>, captured at D = 100,000,000
     (5, 2): {"sources": ["gaf_gram_mma.cuh", "gaf_gramfilter.cuh", "gaf_device.cuh"],
-             "sha256": "86fbf6b03aea3b7b91bdaebc2b2fbc16cf23a7bb73634aaa93d0f7cd31c310c4",
-             "steady": {4: (1604.2e6 + 1170.1e6) / 100e6}},
+             "sha256": "9e4d0496b3660411997f70119a65ea597629d6649e27b79cad70329530722984",
+             "steady": {4: (1604.5e6 + 1169.0e6) / 100e6}},
 }
 
 
@@ -588,8 +588,9 @@ def measure_two_gradients(torch, gaf, workloads, dev, D, steps, nvml, peak, peak
     min_b = (2 * 4 + 4) * D
     out = {"workload": f"gaf_filter_accumulate, K=2, D={D}, f32 inputs ({n_sets} rotating sets)",
            "op": "gaf_filter_accumulate", "unit": UNIT, "min_bytes_per_call": min_b,
-           "byte_model": "both gradients read once, the output written once when the previous call's outcome repeats: "
-                         "(2 b + 4) D (= the minimum); 20 D when it does not", "peak": peak, "peak_kind": peak_kind}
+           "byte_model": "both gradients read once, the output written once when the outcome of the latest two calls "
+                         "repeats: (2 b + 4) D (= the minimum); two passes (16 D or 20 D) while outcomes alternate",
+           "peak": peak, "peak_kind": peak_kind}
     for name, taus in (("all_accepted", (2.0,)), ("all_rejected", (0.0,)), ("alternating", (2.0, 0.0))):
         def step(i, taus=taus):
             gaf.gaf_filter_accumulate(sets[i % n_sets], taus[i % len(taus)], ws, macro_out=macro, mask_out=mask,

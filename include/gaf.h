@@ -108,11 +108,12 @@ enum {
                                    With K = 2 (the setting of the paper's experiments, Section 4) the
                                    result is either the mean of both gradients or the seed alone, and
                                    the first pass writes one of the two while it reads: the one the
-                                   latest such call on the same workspace ended with (a word in the
-                                   workspace; a fresh workspace guesses "both").  A call whose decision
-                                   matches the guess moves (2 b + 4) D bytes and has no second pass; one
-                                   that does not rewrites the output.  The values never depend on the
-                                   guess.  GAF_SCHED_AUTO takes this form for K = 2 at every length. */
+                                   latest two such calls on the same workspace both ended with (a word
+                                   in the workspace; a fresh workspace guesses "both"; no guess while
+                                   the latest two differ).  A call whose decision matches the guess
+                                   moves (2 b + 4) D bytes and has no second pass; one that does not
+                                   rewrites the output.  The values never depend on the guess.
+                                   GAF_SCHED_AUTO takes this form for K = 2 at every length. */
 };
 
 /* Bits of the device status word. */

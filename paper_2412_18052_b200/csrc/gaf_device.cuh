@@ -17,7 +17,7 @@ constexpr int kOct = 8;                 // elements handled per inner step
 // Control block at the start of the caller's workspace.
 struct Control {
     unsigned int ticket;                // last-block election, wraps to 0 by itself
-    unsigned int pair_hint;             // one-launch schedule with two gradients: 1 = the latest such call kept the seed alone
+    unsigned int pair_hint;             // one-launch schedule with two gradients: what the latest two calls kept (0 both, 1 the seed alone, 2 | latest: they differed)
     unsigned int reserved1;
     int status;                         // GAF_STATUS_* bits of the latest call
     int count;                          // running c of Algorithm 1

@@ -106,10 +106,11 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     constexpr int NP = KT * (KT + 1) / 2;
     constexpr int N = FusedVec<T>::N;
     // With two gradients (the paper's own experiments: Section 4) the output can only be the mean of both or the
-    // seed alone, so the first pass writes one of the two while it forms the sums -- the one the latest call on this
-    // workspace ended with (decisions of consecutive training steps go together) -- and the second pass runs
-    // only when this call decides otherwise: 12 bytes per fp32 element instead of 20 (16 for the seed alone) when
-    // the guess holds, 20 when it does not.  The guess changes which stores happen, never their values.
+    // seed alone, so the first pass writes one of the two while it forms the sums -- the one the latest two calls on
+    // this workspace both ended with (decisions of consecutive training steps go together; no guess while they
+    // differ) -- and the second pass runs only when this call decides otherwise: 12 bytes per fp32 element instead
+    // of 20 (16 for the seed alone) when the guess holds, 24 when it does not, the usual 20 / 16 without a guess.
+    // The guess changes which stores happen, never their values.
     constexpr bool kSpeculative = KT == 2;
     extern __shared__ uint4 parked[];       // [round][gradient][thread]
     __shared__ double sacc[kGsThreads / 32][NP];
@@ -134,7 +135,10 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     for (int p = lane; p < NP; p += 32) sacc[warp][p] = 0.0;
     __syncwarp();
     // (read before this CTA arrives, hence before any CTA can have decided and written the next guess)
-    const bool guess_seed_alone = kSpeculative && ld_relaxed_u32(&ctl->pair_hint) != 0;
+    // 0 / 1: the latest two such calls both kept both gradients / the seed alone: write that now;
+    // 2 / 3: they differed (the latest kept both / the seed alone): no guess, two passes as with more gradients
+    const unsigned int hint = kSpeculative ? ld_relaxed_u32(&ctl->pair_hint) : 2u;
+    const bool guessing = hint < 2u, guess_seed_alone = (hint & 1u) != 0;
 
     const T *row[KT];
 #pragma unroll
@@ -181,7 +185,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
             float x[KT][N];
 #pragma unroll
             for (int r = 0; r < KT; ++r) FusedVec<T>::widen(raw[r], x[r]);
-            if constexpr (kSpeculative) {
+            if (kSpeculative && guessing) {
                 // two gradients: the guessed result is written now
                 float v[N];
 #pragma unroll
@@ -207,7 +211,7 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
         float x[KT];
 #pragma unroll
         for (int r = 0; r < KT; ++r) x[r] = load1<T>(row[r], e);
-        if constexpr (kSpeculative) a.out[e] = guess_seed_alone ? x[0] : (x[0] + x[1]) / 2.0f;
+        if (kSpeculative && guessing) a.out[e] = guess_seed_alone ? x[0] : (x[0] + x[1]) / 2.0f;
         int p = 0;
 #pragma unroll
         for (int r = 0; r < KT; ++r)
@@ -275,8 +279,9 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
     // the same division as below).  Otherwise every thread overwrites, below, exactly what it wrote then.
     if constexpr (kSpeculative) {
         const bool seed_alone = n == 1 && list_row[0] == 0;     // (the order-indifferent variant may keep row 1 alone)
-        if (publisher && tid == 0) ctl->pair_hint = n == 1 ? 1u : 0u;
-        if (guess_seed_alone ? seed_alone : n == 2) return;
+        const unsigned int outcome = n == 1 ? 1u : 0u;
+        if (publisher && tid == 0) ctl->pair_hint = outcome == (hint & 1u) ? outcome : (2u | outcome);
+        if (guessing && (guess_seed_alone ? seed_alone : n == 2)) return;
     }
 
     // ---- pass 2a: the rounds that were not parked, last first (what pass 1 read last is what L2 still
