@@ -606,6 +606,46 @@ def measure_two_gradients(torch, gaf, workloads, dev, D, steps, nvml, peak, peak
     return out
 
 
+def measure_variants(torch, gaf, workloads, dev, steps, nvml, peak, peak_kind):
+    """The other forms of the filter at configuration 2 (K=4, D=11,227,812 fp32, tau 0.97, four rotating sets): the
+    order-indifferent variant, the bucketed variant with ResNet18's 62 parameter tensors as buckets, and the
+    streaming form (one call per arriving gradient)."""
+    import numpy as np
+    sets = [workloads.config(2, device=dev, seed=1 + 1000 * i).grads for i in range(4)]
+    K, D = len(sets[0]), sets[0][0].numel()
+    ws = gaf.new_workspace(K, D, gaf.GAF_F32, device=dev)
+    macro = torch.empty(D, dtype=torch.float32, device=dev)
+    bounds = [0] + [int(x) // 8 * 8 for x in np.cumsum(workloads.resnet18_tensor_sizes(100))[:-1]] + [D]
+    bounds = sorted(set(bounds))
+    min_b = (K * 4 + 4) * D
+
+    def any_seed(i):
+        gaf.gaf_filter_accumulate_any_seed(sets[i % 4], 0.97, ws, macro_out=macro)
+
+    def bucketed(i):
+        gaf.gaf_filter_accumulate_bucketed(sets[i % 4], 0.97, bounds, ws, macro_out=macro)
+
+    def streaming(i):
+        g = sets[i % 4]
+        gaf.gaf_stream_begin(g[0], macro, ws)
+        for t in range(1, K):
+            gaf.gaf_stream_push(g[t], t, 0.97, macro, ws)
+        gaf.gaf_stream_end(K, macro, ws)
+
+    out = {"workload": f"configuration 2 recipe, K={K}, D={D}, f32 inputs (4 rotating sets)", "unit": UNIT,
+           "min_bytes_per_call": min_b, "peak": peak, "peak_kind": peak_kind}
+    for name, op, step in (("any_seed", "gaf_filter_accumulate_any_seed", any_seed),
+                           ("bucketed", f"gaf_filter_accumulate_bucketed, {len(bounds) - 1} buckets", bucketed),
+                           ("streaming", "gaf_stream_begin + 3 gaf_stream_push + gaf_stream_end", streaming)):
+        t = timed_region(torch, step, steps, 5, nvml)
+        ms = t["ms_per_step"]
+        out[name] = {"op": op, "steps": steps, "ms_per_call": ms,
+                     "ms_per_call_median_of_event_pairs": statistics.median(t["per_call_ms"]),
+                     "value": K * 4 * D / (ms * 1e-3) / 1e9, "min_bytes_frac": min_b / (ms * 1e-3) / 1e9 / peak,
+                     "clocks": t["clocks"]}
+    return out
+
+
 def pairwise_entry(m, peak, peak_kind, steps):
     t = m["timing"]
     ms = t["ms_per_step"]
@@ -767,6 +807,12 @@ def run_ours(args):
             gc.collect()
             torch.cuda.empty_cache()
 
+        try:
+            block["variants_config2"] = measure_variants(torch, gaf, workloads, dev, 500, nvml, peak, peak_kind)
+        except Exception as exc:
+            block["variants_config2"] = {"error": f"{type(exc).__name__}: {exc}"}
+        gc.collect()
+        torch.cuda.empty_cache()
         for key, D_c, n in (("two_gradients_D11.2M", FULL_D[2], 1000), ("two_gradients_D124M", FULL_D[4], 100)):
             try:
                 block[key] = measure_two_gradients(torch, gaf, workloads, dev, D_c, n, nvml, peak, peak_kind)
