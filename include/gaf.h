@@ -79,9 +79,9 @@ enum {
 enum {
     GAF_SCHED_AUTO = 0,         /* the library picks: Gram-first where a one-pass Gram kernel
                                    pays off (K <= 32; bfloat16: K <= 64), else stepwise.
-                                   For K <= 8 the one-launch form is taken for binary32 inputs of
-                                   at most 512 MB in all, and for bfloat16 inputs except 8
-                                   gradients of more than 1 GB in all (tensor-core Gram then);
+                                   For K <= 8 the one-launch form is taken for K = 2, for binary32
+                                   inputs of at most 512 MB in all, and for bfloat16 inputs except 7
+                                   or 8 gradients of more than 1 GB in all (tensor-core Gram then);
                                    if the device refuses that launch, two launches. */
     GAF_SCHED_STEPWISE = 1,     /* streaming: one launch per step; each launch adds the
                                    gradient accepted at step t to the running sum and, in
@@ -369,8 +369,9 @@ int gaf_last_schedule(void);
  * its tiles: 0 the call did not use that kernel, 1 16-byte asynchronous copies, 2 tensor copies (TMA) --
  * taken when the gradients are rows of one matrix: grads[i] = grads[0] + i * stride with a positive stride
  * that is a multiple of 128 bytes (the layout an all-gather of flattened, padded micro-gradients leaves),
- * 64 <= D < 2^31, at most 52 gradients (beyond that the 16-byte copies measured faster).  About a tenth faster; both give the same Gram matrix up to the rounding order inside
- * one MMA.  Host-side, for tests. */
+ * 64 <= D < 2^31, at most 52 gradients (beyond that the 16-byte copies measured faster).  The tensor
+ * copies are 5 to 10 % faster; both give the same Gram matrix up to the rounding order inside one MMA.
+ * Host-side, for tests. */
 int gaf_last_gram_loader(void);
 
 /*
