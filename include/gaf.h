@@ -101,7 +101,9 @@ enum {
                                    for K > 8.  Such a call needs the whole device for its CTAs to meet:
                                    calls on one stream are ordered and fine; a second one on ANOTHER
                                    stream while the first stream still has work pending returns
-                                   GAF_ERR_UNSUPPORTED (GAF_SCHED_AUTO takes two launches then).  The one
+                                   GAF_ERR_UNSUPPORTED (GAF_SCHED_AUTO takes two launches then), and so
+                                   does a call on a stream that is being captured into a graph (what
+                                   runs beside the node is decided at replay).  The one
                                    wait on other CTAs is bounded: GAF_STATUS_TIMEOUT if it ever runs out
                                    (only when something else, another process say, keeps part of the
                                    device busy for seconds).

@@ -508,6 +508,13 @@ int launch_gram_fused_kt(GramFusedArgs &a, const DeviceInfo &di, cudaStream_t st
     // resident and the one wait on other CTAs ends; it is bounded in any case.  Programmatic stream
     // serialisation: the kernel waits for its predecessor on the stream itself (griddepcontrol.wait, first
     // thing) and releases its successor once its decisions are taken.
+    // Not while the stream is being captured into a graph: where the node will run, and beside what, is decided
+    // at replay, out of this library's sight (and the query below is not allowed during a capture).
+    {
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &capturing) != cudaSuccess) { cudaGetLastError(); return GAF_ERR_CUDA; }
+        if (capturing != cudaStreamCaptureStatusNone) return GAF_ERR_UNSUPPORTED;
+    }
     FusedGuard &guard = g_fused_guard[di.dev];
     std::lock_guard<std::mutex> lock(guard.m);          // (check and launch are one step for other host threads)
     if (guard.any && guard.last != st) {

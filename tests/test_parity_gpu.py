@@ -281,6 +281,46 @@ def test_one_launch_calls_do_not_overlap_across_streams(ws):
     check_filter(w.grads, 0.9, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED)
 
 
+def test_calls_captured_into_a_graph(ws):
+    """Calls made while the stream is being captured into a CUDA graph: the library's own choice takes the forms
+    that need no co-resident grid (two launches), an explicit request for the one-launch form is refused, and
+    replaying the graph on new inputs (same buffers) gives what the oracle gives."""
+    from oracle import gaf_oracle as orc
+    cases = [(4, 300_007, "f32"), (2, 100_003, "f32"), (8, 200_001, "bf16"), (32, 70_001, "bf16")]
+    for K, D, dtype in cases:
+        w = _mix(K, D, dtype, seed=40 + K)
+        macro = torch.empty(D, dtype=torch.float32, device="cuda")
+        mask = torch.empty(K, dtype=torch.uint8, device="cuda")
+        dist = torch.empty(K, dtype=torch.float32, device="cuda")
+        count = torch.empty(1, dtype=torch.int32, device="cuda")
+        args = dict(macro_out=macro, mask_out=mask, dist_out=dist, count_out=count)
+        gaf.gaf_filter_accumulate(w.grads, 0.97, ws, **args)            # plans and attributes outside the capture
+        gaf.gaf_filter_accumulate(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM, **args)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            gaf.gaf_filter_accumulate(w.grads, 0.97, ws, **args)
+            assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM, (K, gaf.gaf_last_schedule())
+            if K <= 8:
+                with pytest.raises(gaf.GafError):
+                    gaf.gaf_filter_accumulate(w.grads, 0.97, ws, schedule=gaf.GAF_SCHED_GRAM_FUSED, **args)
+        other = _mix(K, D, dtype, seed=90 + K)
+        for g, o in zip(w.grads, other.grads):
+            g.copy_(o)
+        macro.fill_(7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        want = orc.filter_accumulate([workloads.as_numpy_bits(g) for g in w.grads], 0.97)
+        assert mask.cpu().numpy().tolist() == want.mask.tolist() and int(count.item()) == want.count
+        assert float(np.max(np.abs(dist.cpu().numpy() - want.dist))) < 1e-5
+        got = macro.cpu().numpy().astype(np.float64)
+        assert float(np.linalg.norm(got - want.out) / np.linalg.norm(want.out)) < (1e-6 if dtype == "f32" else 1e-3)
+        # and outside a capture the one-launch form is back
+        gaf.gaf_filter_accumulate(w.grads, 0.97, ws, **args)
+        if K <= 8:
+            assert gaf.gaf_last_schedule() == gaf.GAF_SCHED_GRAM_FUSED
+
+
 def test_filter_random_cases(ws):
     """Seeded random shapes, thresholds, orders and schedules against the oracle."""
     rng = np.random.RandomState(2024)
