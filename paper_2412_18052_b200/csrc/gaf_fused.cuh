@@ -168,42 +168,57 @@ gram_fused_kernel(const __grid_constant__ GramFusedArgs a) {
 
     const int64_t tail0 = n_vec * N;
     // ---- pass 1: Gram partial sums; the first rounds stay in shared memory ----
+    // (with two gradients a thread would have only two 16-byte loads in flight: it fetches two rounds at a time;
+    // the rounds are still consumed in order, so the sums are the same)
+    constexpr int U1 = KT <= 2 ? 2 : 1;
     int since_flush = 0;
-    for (int64_t j = 0; j < rounds; ++j) {
-        const int64_t q = warp_first + j * stride + lane;
-        if (q < n_vec) {
-            const bool park = j < parked_rounds;
-            const uint64_t pol = (q * N >= a.keep_from) ? pol_last : pol_first;
-            uint4 raw[KT];
+    for (int64_t j0 = 0; j0 < rounds; j0 += U1) {
+        int64_t q[U1];
+        bool ok[U1];
+        uint4 raw[U1][KT];
 #pragma unroll
-            for (int r = 0; r < KT; ++r) raw[r] = ld16_policy(row[r] + q * N, pol);
-            if (park) {
-                uint4 *slot = parked + (size_t)j * KT * kGsThreads + tid;
+        for (int u = 0; u < U1; ++u) {
+            q[u] = warp_first + (j0 + u) * stride + lane;
+            ok[u] = j0 + u < rounds && q[u] < n_vec;
+            if (ok[u]) {
+                const uint64_t pol = (q[u] * N >= a.keep_from) ? pol_last : pol_first;
 #pragma unroll
-                for (int r = 0; r < KT; ++r) slot[r * kGsThreads] = raw[r];
+                for (int r = 0; r < KT; ++r) raw[u][r] = ld16_policy(row[r] + q[u] * N, pol);
             }
-            float x[KT][N];
-#pragma unroll
-            for (int r = 0; r < KT; ++r) FusedVec<T>::widen(raw[r], x[r]);
-            if (kSpeculative && guessing) {
-                // two gradients: the guessed result is written now
-                float v[N];
-#pragma unroll
-                for (int k = 0; k < N; ++k) v[k] = guess_seed_alone ? x[0][k] : (x[0][k] + x[1][k]) / 2.0f;
-                store_vec_streaming<N>(a.out + q * N, v);
-            }
-            int p = 0;
-#pragma unroll
-            for (int r = 0; r < KT; ++r)
-#pragma unroll
-                for (int c = r; c < KT; ++c, ++p) {
-                    Acc s = acc[p];
-#pragma unroll
-                    for (int k = 0; k < N; ++k) s = gs_fma(x[r][k], x[c][k], s);
-                    acc[p] = s;
-                }
         }
-        if (GsAcc<T, KT>::kPeriodicFlush && ++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+#pragma unroll
+        for (int u = 0; u < U1; ++u) {
+            const int64_t j = j0 + u;
+            if (j >= rounds) break;
+            if (ok[u]) {
+                if (j < parked_rounds) {
+                    uint4 *slot = parked + (size_t)j * KT * kGsThreads + tid;
+#pragma unroll
+                    for (int r = 0; r < KT; ++r) slot[r * kGsThreads] = raw[u][r];
+                }
+                float x[KT][N];
+#pragma unroll
+                for (int r = 0; r < KT; ++r) FusedVec<T>::widen(raw[u][r], x[r]);
+                if (kSpeculative && guessing) {
+                    // two gradients: the guessed result is written now
+                    float v[N];
+#pragma unroll
+                    for (int k = 0; k < N; ++k) v[k] = guess_seed_alone ? x[0][k] : (x[0][k] + x[1][k]) / 2.0f;
+                    store_vec_streaming<N>(a.out + q[u] * N, v);
+                }
+                int p = 0;
+#pragma unroll
+                for (int r = 0; r < KT; ++r)
+#pragma unroll
+                    for (int c = r; c < KT; ++c, ++p) {
+                        Acc s = acc[p];
+#pragma unroll
+                        for (int k = 0; k < N; ++k) s = gs_fma(x[r][k], x[c][k], s);
+                        acc[p] = s;
+                    }
+            }
+            if (GsAcc<T, KT>::kPeriodicFlush && ++since_flush == kGsFlushEvery) { flush(); since_flush = 0; }
+        }
     }
     // ragged tail (D mod N elements), first CTA
     if (blockIdx.x == 0 && tail0 + tid < a.D) {
