@@ -72,6 +72,9 @@ def parse_args():
     ap.add_argument("--fp32", action="store_true", help="pairwise workload only: binary32 inputs (same recipe)")
     ap.add_argument("--separate", action="store_true",
                     help="pairwise workload only: K separate allocations instead of the rows of one matrix")
+    ap.add_argument("--two-gradients", action="store_true",
+                    help="instead of a named configuration: the filter on two fp32 gradients of configuration 2's "
+                         "recipe (the setting of the paper's experiments); --D for another length")
     ap.add_argument("--tau", type=float, default=0.97)
     ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2, 3],
                     help="0 auto, 1 stepwise (streaming), 2 Gram-first in two launches, 3 Gram-first in one launch")
@@ -883,10 +886,46 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_two_gradients(args):
+    """--two-gradients: the K = 2 lines of the configs block alone (one GPU), the repeating-outcome stream as the
+    headline value."""
+    import torch
+
+    import paper_2412_18052_b200 as gaf
+    from paper_2412_18052_b200 import workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(0)
+    nvml = Nvml(0)
+    peak, peak_kind = peak_bandwidth()
+    D = args.D or FULL_D[2]
+    m = measure_two_gradients(torch, gaf, workloads, "cuda:0", D, args.steps, nvml, peak, peak_kind)
+    head = m["all_accepted"]
+    line = {
+        "metric": "gaf_filter_accumulate micro-gradient GB/s", "value": head["value"], "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": head["ms_per_call"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 products, f64 sums",
+        "data": "synthetic",
+        "config": {"workload": m["workload"] + " (NOT a named configuration: two gradients, as in the paper's "
+                               "experiments); headline = the stream of calls that all accept"},
+        "roofline": {"bound": "hbm", "achieved": head["min_bytes_frac"] * peak, "peak": peak, "unit": "GB/s",
+                     "frac": head["min_bytes_frac"], "basis": "min_bytes: (2 b + 4) D", "traffic": None,
+                     "peak_kind": peak_kind, "kernel": "gram_fused_kernel<float, 2>",
+                     "algorithmic_bytes_per_launch": m["min_bytes_per_call"]},
+        "two_gradients": m, "e2e": None, "gpu_launches": head["launches_per_call"] * args.steps,
+        "clocks": head["clocks"], "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.two_gradients:
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_two_gradients(args)
     elif args.workload == 3:
         if int(os.environ.get("RANK", "0")) == 0:
             run_pairwise(args)
