@@ -308,7 +308,7 @@ int gaf_filter_accumulate_host(const void *const *grads_host, int K, int64_t D, 
  *   dist_out    device, K*K floats row-major; symmetric; diagonal 0 (1 for a
  *               zero-norm gradient, whose whole row and column are 1)
  *   gram_out    device, K*K doubles row-major (the Gram matrix); may be NULL
- * bfloat16 with 17 to 52 gradients runs fastest when the gradients are rows of one matrix (see
+ * bfloat16 with 17 to 42 gradients runs fastest when the gradients are rows of one matrix (see
  * gaf_last_gram_loader); any other placement is accepted.
  */
 int gaf_pairwise_cosdist(const void *const *grads, int K, int64_t D, int dtype,
@@ -371,8 +371,10 @@ int gaf_last_schedule(void);
  * its tiles: 0 the call did not use that kernel, 1 16-byte asynchronous copies, 2 tensor copies (TMA) --
  * taken when the gradients are rows of one matrix: grads[i] = grads[0] + i * stride with a positive stride
  * that is a multiple of 128 bytes (the layout an all-gather of flattened, padded micro-gradients leaves),
- * 64 <= D < 2^31, at most 52 gradients (beyond that the 16-byte copies measured faster).  The tensor
- * copies are 5 to 10 % faster; both give the same Gram matrix up to the rounding order inside one MMA.
+ * 64 <= D < 2^31, at most 42 gradients (beyond that the 16-byte copies measured faster).  The tensor
+ * copies are 5 % faster at 32 gradients and up to 47 % where the gradients do not fill a power of two (17..25,
+ * 33..42: they stack floor(128 / K) chunks of the vector in a tile instead of 128 / 32 or 128 / 64); both give
+ * the same Gram matrix up to the rounding order inside one MMA.
  * Host-side, for tests. */
 int gaf_last_gram_loader(void);
 

@@ -203,7 +203,7 @@ TensorMapEncodeFn tensor_map_encoder() {
     return reinterpret_cast<TensorMapEncodeFn>(fn.load(std::memory_order_relaxed));
 }
 
-constexpr int kTcTensorCopyMaxWideK = 52;
+constexpr int kTcTensorCopyMaxWideK = 42;
 
 #ifndef GAF_TC_L2_PROMOTION
 #define GAF_TC_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_128B
@@ -212,15 +212,16 @@ constexpr int kTcTensorCopyMaxWideK = 52;
 // The K bfloat16 gradients as one tensor for tensor copies: possible when they are rows of one matrix (equal,
 // positive distances between their addresses, multiples of 128 bytes), at least one whole 64-element chunk long,
 // and every element coordinate a tile can ask for fits 32 bits.  `tile_map` sees {64 elements, D / 64 chunks, K
-// gradients} and copies boxes of {64, R, Kp}: R consecutive chunks (R x 128 contiguous bytes) of each gradient;
+// gradients} and copies boxes of {64, R, K}: R consecutive chunks (R x 128 contiguous bytes) of each gradient;
 // `row_map` sees {D elements, K gradients} and copies one 64-element row at a time (the ragged last chunk).  Both
 // with the 128-byte swizzle; what lies outside reads as zero.
-bool stacked_tensor_maps(const void *const *grads, int K, int Kp, int64_t D, int64_t tile_elems, CUtensorMap *tile_map,
-                         CUtensorMap *row_map) {
+bool stacked_tensor_maps(const void *const *grads, int K, int Kp, int R, int box_k, int64_t D, int64_t tile_elems,
+                         CUtensorMap *tile_map, CUtensorMap *row_map) {
     if (K < 2 || Kp < 32 || D < 64 || !aligned16(grads[0])) return false;
-    // 64-row-pair tiles (33..64 gradients) give a box only 256 contiguous bytes per gradient, and the copy engine's
-    // rate falls with the number of separate pieces: measured at D = 11.2 M against the 16-byte copies, 195 / 227 us
-    // against 210 / 238 us at 40 / 52 gradients, but 252 / 272 / 292 against 243 / 250 / 259 us at 56 / 60 / 64.
+    // From 43 gradients on only two chunks fit the 128 rows, a box then has 256 contiguous bytes per gradient, and
+    // the copy engine's rate falls with the number of separate pieces: measured at D = 11.2 M against the 16-byte
+    // copies, 228 / 240 / 252 us against 219 / 228 / 236 us at 44 / 48 / 52 gradients (three chunks, up to 42
+    // gradients: 149 / 170 us against 204 / 224 us at 33 / 40).
     if (Kp == 64 && K > kTcTensorCopyMaxWideK) return false;
     const intptr_t base = reinterpret_cast<intptr_t>(grads[0]);
     const intptr_t stride = reinterpret_cast<intptr_t>(grads[1]) - base;
@@ -234,7 +235,7 @@ bool stacked_tensor_maps(const void *const *grads, int K, int Kp, int64_t D, int
     {
         const cuuint64_t dims[3] = {64u, cuuint64_t(D / 64), cuuint64_t(K)};
         const cuuint64_t strides[2] = {128u, cuuint64_t(stride)};
-        const cuuint32_t box[3] = {64u, cuuint32_t(128 / Kp), cuuint32_t(Kp)};
+        const cuuint32_t box[3] = {64u, cuuint32_t(R), cuuint32_t(box_k)};
         const cuuint32_t elem_strides[3] = {1u, 1u, 1u};
         if (encode(tile_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, origin, dims, strides, box, elem_strides,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, GAF_TC_L2_PROMOTION,
@@ -291,18 +292,22 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         for (int i = 0; i < K; ++i) t.g[i] = grads[i];
         t.K = K; t.Kp = K <= 8 ? 8 : (K <= 16 ? 16 : (K <= 32 ? 32 : 64)); t.D = D;
         t.partials = a.partials; t.tiles = a.tiles; t.ctl = a.ctl;
-        const int64_t unit = (128 / t.Kp) * 64 * kTcSub;
-        const int64_t units = (D + unit - 1) / unit;
-        int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;
-        if (slices > units) slices = units;
-        if (slices < 1) slices = 1;
-        a.slices = int(slices);
         const int dyn = kTcStages * kTcStageBytes + 1024;
         // gradients that are rows of one matrix are fetched by tensor copies, any others by 16-byte copies
         alignas(64) CUtensorMap tmap, tmap_row;
         std::memset(&tmap, 0, sizeof tmap);
         std::memset(&tmap_row, 0, sizeof tmap_row);
-        const bool tma = stacked_tensor_maps(grads, K, t.Kp, D, unit, &tmap, &tmap_row);
+        // (tensor copies stack floor(128 / K) chunks of D in the 128 rows, the 16-byte copies 128 / Kp)
+        t.R = 128 / K;
+        t.box_k = t.R == 128 / t.Kp ? t.Kp : K;
+        const int64_t unit_tma = int64_t(t.R) * 64 * kTcSub;
+        const bool tma = stacked_tensor_maps(grads, K, t.Kp, t.R, t.box_k, D, unit_tma, &tmap, &tmap_row);
+        const int64_t unit = tma ? unit_tma : int64_t(128 / t.Kp) * 64 * kTcSub;   // elements of D per tile
+        const int64_t units = (D + unit - 1) / unit;
+        int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;
+        if (slices > units) slices = units;
+        if (slices < 1) slices = 1;
+        a.slices = int(slices);
         g_gram_loader = tma ? 2 : 1;
         void (*kernel)(GramTcArgs, CUtensorMap, CUtensorMap) =
             t.Kp == 64 ? (tma ? gram_tc_kernel<true, true> : gram_tc_kernel<true, false>)

@@ -45,6 +45,8 @@
 // finishing kernel totals the slices.  Every wait is bounded.
 #pragma once
 
+#include <type_traits>
+
 #include <cuda.h>        // CUtensorMap (the type only: the encoder is fetched from the driver at run time)
 
 #include "gaf_device.cuh"
@@ -76,6 +78,8 @@ struct GramTcArgs {
     const void *g[kTcMaxK];
     int K;                  // gradients
     int Kp;                 // 8, 16, 32 or 64
+    int R;                  // tensor-copy form: chunks of D stacked in the 128 rows, floor(128 / K) (2..7)
+    int box_k;              // tensor-copy form: gradients a box covers (K, or Kp when that stacks as many chunks)
     int64_t D;
     double *partials;       // [tile pair][slice][64]
     int tiles;              // ceil(K / 8)
@@ -225,7 +229,7 @@ struct GramTcShared {
 // the tensor-memory lanes 32 (warp mod 4) .. + 31) takes the upper 32 columns of each block.
 //
 // TMA: the tiles are filled by tensor copies, gradient-major rows (Kp is 32 or 64 then): `tmap` has the
-// dimensions {64, D / 64, K} of bfloat16 and the box {64, R, Kp}, `tmap_row` the dimensions {D, K} and the box
+// dimensions {64, D / 64, K} of bfloat16 and the box {64, R, K}, `tmap_row` the dimensions {D, K} and the box
 // {64, 1}; both with the 128-byte swizzle and zero fill outside.  Otherwise neither map is touched.
 // Threads of a launch: four epilogue warps, the loader warps (one with tensor copies), the MMA warp, and four
 // more epilogue warps for 33..64 gradients.
@@ -247,7 +251,10 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     const uint32_t tiles_u32 = tc_smem_u32(tiles);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int K = a.K, Kp = a.Kp, R = 128 / Kp;
+    // Chunks of D stacked in the rows.  The 16-byte-copy form pads the gradients to Kp, so that a chunk's partial
+    // Gram matrix is a diagonal block; the tensor-copy form needs no such padding (its epilogue picks single
+    // columns) and stacks as many chunks as fit: 7 with 17 or 18 gradients, 3 with 33 to 42.
+    const int K = a.K, Kp = a.Kp, R = TMA ? a.R : 128 / Kp;
     const int64_t unit = (int64_t)R * 64 * kTcSub;       // elements of D per tile and gradient
     // the last tile may be partial: its missing elements are zero-filled by the copies
     const int64_t n_units = (a.D + unit - 1) / unit;
@@ -271,11 +278,12 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // rows of absent gradients (K < Kp) stay zero for the whole kernel (the tensor copies write them as zeros)
-    if (!TMA && K < Kp) {
+    // rows that no copy ever writes stay zero for the whole kernel: those of absent gradients (K < Kp), or, with
+    // tensor copies, the rows past the K R that a box fills
+    if (TMA ? a.box_k * R < 128 : K < Kp) {
         for (int idx = threadIdx.x; idx < kTcStages * kTcSub * 128 * 8; idx += kThreads) {
             const int row = (idx >> 3) & 127;
-            if ((row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
+            if (TMA ? row >= a.box_k * R : (row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
         }
         tc_fence_async_smem();
     }
@@ -319,7 +327,7 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
                     break;
                 const int64_t elem0 = (blockIdx.x + it * G) * unit;   // first element of the tile, per gradient
                 const uint32_t tile = tiles_u32 + (uint32_t)s * kTcStageBytes;
-                if (lane == 0) tc_mbar_arrive_expect_tx(&sh.full[s], (uint32_t)kTcStageBytes);
+                if (lane == 0) tc_mbar_arrive_expect_tx(&sh.full[s], (uint32_t)(kTcSub * a.box_k * R * 128));
                 __syncwarp();
                 for (int b = 0; b < kTcSub; ++b) {
                     // block b: chunks chunk0 .. chunk0 + R - 1 of every gradient, row i R + c
@@ -329,9 +337,9 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
                         if (lane == 0) tc_tma_load_3d(block, &tmap, 0, (int32_t)chunk0, 0, &sh.full[s]);
                     } else {
                         // the one block of the whole vector that holds the partial last chunk: row by row through
-                        // the element-granular map, which fills what lies past D (and past K) with zeros; the
-                        // lanes issue four rows each (one thread issuing all 128 took 5 us)
-                        for (int row = lane; row < 128; row += 32)
+                        // the element-granular map, which fills what lies past D with zeros; the lanes issue
+                        // up to four rows each (one thread issuing all of them took 5 us)
+                        for (int row = lane; row < a.box_k * R; row += 32)
                             tc_tma_load_2d(block + (uint32_t)row * 128u, &tmap_row,
                                            (int32_t)((chunk0 + row % R) * 64), row / R, &sh.full[s]);
                     }
@@ -439,44 +447,68 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
         __syncwarp();
     } else {
         // ------------------------------------------------------ epilogue -------
-        for (int blk = 0; blk < n_blocks; ++blk) {
-            const int buf = blk & 1;
-            // (warp-uniform outcome: the load below needs the whole warp)
-            if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag, a.spin_limit)) break;
-            tc_fence_after_sync();
-            uint32_t r[32];
-            const uint32_t taddr = tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128 + epi_col0);
-            if constexpr (!TMA) {
-                tc_tmem_ld32(taddr, r);
+        if constexpr (!TMA) {
+            for (int blk = 0; blk < n_blocks; ++blk) {
+                const int buf = blk & 1;
+                // (warp-uniform outcome: the load below needs the whole warp)
+                if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag, a.spin_limit)) break;
+                tc_fence_after_sync();
+                uint32_t r[32];
+                tc_tmem_ld32(tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128 + epi_col0), r);
                 tc_fence_before_sync();
                 tc_mbar_arrive(&sh.acc_empty[buf]);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) gsum[j] += (double)__uint_as_float(r[j]);
-            } else {
-                // this row holds chunk c of its gradient: its Gram entries are the columns j R + c
-                constexpr int RR = WIDE ? 2 : 4;             // R
-                constexpr int kPer = 32 / RR;                // gradients per 32 loaded columns
-                const int c = lane & (RR - 1);
+            }
+        } else {
+            // Gradient-major rows: this row holds chunk c of its gradient, its Gram entries are the columns j R + c.
+            // All 128 columns are read, 32 at a time, and every row keeps, per gradient j, the column of its own
+            // chunk (one select per column; j and the column's chunk are compile-time), then adds those.  RR = R,
+            // J0 = the first of the 32 gradients this warp set keeps.
+            const int c = (epi_q * 32 + lane) % R;
+            auto drain_all = [&](auto rr_tag, auto j0_tag) {
+                constexpr int RR = decltype(rr_tag)::value, J0 = decltype(j0_tag)::value;
+                for (int blk = 0; blk < n_blocks; ++blk) {
+                    const int buf = blk & 1;
+                    if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag, a.spin_limit)) break;
+                    tc_fence_after_sync();
+                    const uint32_t taddr = tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128);
+                    uint32_t sel[32];                        // the column of this row's chunk, per gradient
 #pragma unroll
-                for (int t = 0; t < RR; ++t) {
-                    tc_tmem_ld32(taddr + (uint32_t)(32 * t), r);
-                    if (t == RR - 1) {
-                        tc_fence_before_sync();
-                        tc_mbar_arrive(&sh.acc_empty[buf]);
-                    }
+                    for (int j = 0; j < 32; ++j) sel[j] = 0u;
 #pragma unroll
-                    for (int jj = 0; jj < kPer; ++jj) {
-                        uint32_t v;
-                        if constexpr (WIDE) {
-                            v = c ? r[2 * jj + 1] : r[2 * jj];
-                        } else {
-                            const uint32_t lo = (c & 1) ? r[4 * jj + 1] : r[4 * jj];
-                            const uint32_t hi = (c & 1) ? r[4 * jj + 3] : r[4 * jj + 2];
-                            v = (c & 2) ? hi : lo;
+                    for (int t = 0; t < 4; ++t) {
+                        // (a batch none of whose columns belongs to this warp set's gradients is not read)
+                        if ((32 * t + 31) / RR < J0 || (32 * t) / RR >= J0 + 32) continue;
+                        uint32_t r[32];
+                        tc_tmem_ld32(taddr + (uint32_t)(32 * t), r);
+#pragma unroll
+                        for (int n = 0; n < 32; ++n) {
+                            const int col = 32 * t + n;
+                            const int j = col / RR, cc = col % RR;
+                            if (j >= J0 && j < J0 + 32) sel[j - J0] = (cc == c) ? r[n] : sel[j - J0];
                         }
-                        gsum[t * kPer + jj] += (double)__uint_as_float(v);
                     }
+                    tc_fence_before_sync();
+                    tc_mbar_arrive(&sh.acc_empty[buf]);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) gsum[j] += (double)__uint_as_float(sel[j]);
                 }
+            };
+            using std::integral_constant;
+            const bool upper = WIDE && warp > kMmaWarp;
+            if (!upper) {
+                switch (R) {
+                    case 2: drain_all(integral_constant<int, 2>(), integral_constant<int, 0>()); break;
+                    case 3: drain_all(integral_constant<int, 3>(), integral_constant<int, 0>()); break;
+                    case 4: drain_all(integral_constant<int, 4>(), integral_constant<int, 0>()); break;
+                    case 5: drain_all(integral_constant<int, 5>(), integral_constant<int, 0>()); break;
+                    case 6: drain_all(integral_constant<int, 6>(), integral_constant<int, 0>()); break;
+                    default: drain_all(integral_constant<int, 7>(), integral_constant<int, 0>()); break;
+                }
+            } else {
+                if (R == 2) drain_all(integral_constant<int, 2>(), integral_constant<int, 32>());
+                else drain_all(integral_constant<int, 3>(), integral_constant<int, 32>());
             }
         }
     }
@@ -495,7 +527,7 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     // the streaming part of this CTA is over: the finishing kernel, launched as a programmatic
     // dependent, may be placed now; it still waits for this whole grid before it reads the partials
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles <= 64 KB)
+    // the tile ring is idle now: reuse it as red[c][i][j] (R * Kp * Kp doubles, at most 96 KB)
     double *red = reinterpret_cast<double *>(tiles);
     if (warp < 4 || warp > kMmaWarp) {
         const int row = epi_q * 32 + lane;               // row of the 128 x 128 result
