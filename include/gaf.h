@@ -372,9 +372,8 @@ int gaf_last_schedule(void);
  * taken when the gradients are rows of one matrix: grads[i] = grads[0] + i * stride with a positive stride
  * that is a multiple of 128 bytes (the layout an all-gather of flattened, padded micro-gradients leaves),
  * 64 <= D < 2^31, at most 42 gradients (beyond that the 16-byte copies measured faster).  The tensor
- * copies are 5 % faster at 32 gradients and up to 47 % where the gradients do not fill a power of two (17..25,
- * 33..42: they stack floor(128 / K) chunks of the vector in a tile instead of 128 / 32 or 128 / 64); both give
- * the same Gram matrix up to the rounding order inside one MMA.
+ * copies are 3 to 10 % faster up to 32 gradients and 20 to 27 % with 33 to 42; both give the same Gram matrix
+ * up to the rounding order inside one MMA.
  * Host-side, for tests. */
 int gaf_last_gram_loader(void);
 

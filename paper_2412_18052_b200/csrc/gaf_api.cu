@@ -302,7 +302,11 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         t.box_k = t.R == 128 / t.Kp ? t.Kp : K;
         const int64_t unit_tma = int64_t(t.R) * 64 * kTcSub;
         const bool tma = stacked_tensor_maps(grads, K, t.Kp, t.R, t.box_k, D, unit_tma, &tmap, &tmap_row);
-        const int64_t unit = tma ? unit_tma : int64_t(128 / t.Kp) * 64 * kTcSub;   // elements of D per tile
+        // the 16-byte copies write the same gradient-major rows where those stack more chunks per tile than the padded
+        // order (17..25 and 33..42 gradients); elsewhere the padded order's epilogue is the cheaper one
+        const bool gm = tma || 128 / K > 128 / t.Kp;
+        if (!gm) t.R = 128 / t.Kp;
+        const int64_t unit = int64_t(t.R) * 64 * kTcSub;   // elements of D per tile
         const int64_t units = (D + unit - 1) / unit;
         int64_t slices = sms < kGramMaxSlices ? sms : kGramMaxSlices;
         if (slices > units) slices = units;
@@ -310,11 +314,13 @@ int launch_gram_tiles(const void *const *grads, int K, int64_t D, int dtype, flo
         a.slices = int(slices);
         g_gram_loader = tma ? 2 : 1;
         void (*kernel)(GramTcArgs, CUtensorMap, CUtensorMap) =
-            t.Kp == 64 ? (tma ? gram_tc_kernel<true, true> : gram_tc_kernel<true, false>)
-                       : (tma ? gram_tc_kernel<false, true> : gram_tc_kernel<false, false>);
+            t.Kp == 64 ? (tma ? gram_tc_kernel<true, true, true>
+                              : (gm ? gram_tc_kernel<true, false, true> : gram_tc_kernel<true, false, false>))
+                       : (tma ? gram_tc_kernel<false, true, true>
+                              : (gm ? gram_tc_kernel<false, false, true> : gram_tc_kernel<false, false, false>));
         {
-            static PerDevice<DynSmemPlan> table[4];
-            const int w = (t.Kp == 64 ? 1 : 0) + (tma ? 2 : 0);
+            static PerDevice<DynSmemPlan> table[6];
+            const int w = (t.Kp == 64 ? 1 : 0) + (tma ? 2 : 0) + (gm && !tma ? 4 : 0);
             if (int rc = plan_once(table[w].plan[di.dev], table[w].ready[di.dev], [&](DynSmemPlan &pl) {
                     pl.dyn = dyn;
                     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) == cudaSuccess

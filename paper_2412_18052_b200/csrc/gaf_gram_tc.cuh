@@ -236,7 +236,9 @@ struct GramTcShared {
 __host__ __device__ constexpr int tc_mma_warp(bool tma) { return 4 + (tma ? 1 : kTcLoaderWarps); }
 __host__ __device__ constexpr int tc_threads(bool wide, bool tma) { return (tc_mma_warp(tma) + 1) * 32 + (wide ? 128 : 0); }
 
-template <bool WIDE, bool TMA>
+// GM: gradient-major rows (always with tensor copies; with 16-byte copies up to 42 gradients, where they stack more
+// chunks than the padded chunk-major order).
+template <bool WIDE, bool TMA, bool GM>
 __global__ void __launch_bounds__(tc_threads(WIDE, TMA), 1)
 gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUtensorMap tmap,
                const __grid_constant__ CUtensorMap tmap_row) {
@@ -254,7 +256,9 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     // Chunks of D stacked in the rows.  The 16-byte-copy form pads the gradients to Kp, so that a chunk's partial
     // Gram matrix is a diagonal block; the tensor-copy form needs no such padding (its epilogue picks single
     // columns) and stacks as many chunks as fit: 7 with 17 or 18 gradients, 3 with 33 to 42.
-    const int K = a.K, Kp = a.Kp, R = TMA ? a.R : 128 / Kp;
+    static_assert(GM || !TMA, "tensor copies write gradient-major rows");
+    const int K = a.K, Kp = a.Kp, R = GM ? a.R : 128 / Kp;
+    const int rows_filled = TMA ? a.box_k * R : K * R;     // gradient-major: rows that the copies write
     const int64_t unit = (int64_t)R * 64 * kTcSub;       // elements of D per tile and gradient
     // the last tile may be partial: its missing elements are zero-filled by the copies
     const int64_t n_units = (a.D + unit - 1) / unit;
@@ -280,10 +284,10 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     }
     // rows that no copy ever writes stay zero for the whole kernel: those of absent gradients (K < Kp), or, with
     // tensor copies, the rows past the K R that a box fills
-    if (TMA ? a.box_k * R < 128 : K < Kp) {
+    if (GM ? rows_filled < 128 : K < Kp) {
         for (int idx = threadIdx.x; idx < kTcStages * kTcSub * 128 * 8; idx += kThreads) {
             const int row = (idx >> 3) & 127;
-            if (TMA ? row >= a.box_k * R : (row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
+            if (GM ? row >= rows_filled : (row % Kp) >= K) reinterpret_cast<uint4 *>(tiles)[idx] = make_uint4(0, 0, 0, 0);
         }
         tc_fence_async_smem();
     }
@@ -307,7 +311,7 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     // the columns that hold the rows' diagonal block(s): the 32 on the diagonal, or one half of the 64
     // (gradient-major rows: the first of all 128 columns, or of the half that holds this warp set's 32 gradients)
     const int epi_q = warp & 3;
-    const int epi_col0 = TMA ? ((WIDE && warp > kMmaWarp) ? 64 : 0)
+    const int epi_col0 = GM ? ((WIDE && warp > kMmaWarp) ? 64 : 0)
                              : (WIDE ? (epi_q >> 1) * 64 + (warp > kMmaWarp ? 32 : 0) : epi_q * 32);
     double gsum[32];                                     // epilogue: this row's 32 loaded columns
 #pragma unroll
@@ -375,7 +379,7 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
                 const int i = p / run, rem = p % run;
                 const int q = rem >> 3, j = rem & 7;     // 64-element chunk within the run, piece within it
                 const int blk = q / R, c = q % R;        // which swizzle block, which row group
-                const int row = c * Kp + i;
+                const int row = GM ? i * R + c : c * Kp + i;
                 rel_elem[k] = q * 64 + j * 8;
                 src_base[k] = static_cast<const unsigned char *>(a.g[i]) + (int64_t)rel_elem[k] * 2;
                 dst_off[k] = (uint32_t)(blk * kTcBlockBytes + row * 128 + ((j ^ (row & 7)) << 4));
@@ -447,7 +451,7 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
         __syncwarp();
     } else {
         // ------------------------------------------------------ epilogue -------
-        if constexpr (!TMA) {
+        if constexpr (!GM) {
             for (int blk = 0; blk < n_blocks; ++blk) {
                 const int buf = blk & 1;
                 // (warp-uniform outcome: the load below needs the whole warp)
@@ -466,49 +470,55 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
             // chunk (one select per column; j and the column's chunk are compile-time), then adds those.  RR = R,
             // J0 = the first of the 32 gradients this warp set keeps.
             const int c = (epi_q * 32 + lane) % R;
-            auto drain_all = [&](auto rr_tag, auto j0_tag) {
-                constexpr int RR = decltype(rr_tag)::value, J0 = decltype(j0_tag)::value;
+            auto drain_all = [&](auto rr_tag, auto j0_tag, auto nj_tag) {
+                // NJ: how many gradients, from J0 on, this warp set keeps (what is never indexed costs no register)
+                constexpr int RR = decltype(rr_tag)::value, J0 = decltype(j0_tag)::value, NJ = decltype(nj_tag)::value;
                 for (int blk = 0; blk < n_blocks; ++blk) {
                     const int buf = blk & 1;
                     if (!tc_mbar_wait_warp(&sh.acc_full[buf], (uint32_t)((blk / 2) & 1), &sh.abort_flag, a.spin_limit)) break;
                     tc_fence_after_sync();
                     const uint32_t taddr = tmem_base + ((uint32_t)(epi_q * 32) << 16) + (uint32_t)(buf * 128);
-                    uint32_t sel[32];                        // the column of this row's chunk, per gradient
+                    uint32_t sel[NJ];                        // the column of this row's chunk, per gradient
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) sel[j] = 0u;
+                    for (int j = 0; j < NJ; ++j) sel[j] = 0u;
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
                         // (a batch none of whose columns belongs to this warp set's gradients is not read)
-                        if ((32 * t + 31) / RR < J0 || (32 * t) / RR >= J0 + 32) continue;
+                        if ((32 * t + 31) / RR < J0 || (32 * t) / RR >= J0 + NJ) continue;
                         uint32_t r[32];
                         tc_tmem_ld32(taddr + (uint32_t)(32 * t), r);
 #pragma unroll
                         for (int n = 0; n < 32; ++n) {
                             const int col = 32 * t + n;
                             const int j = col / RR, cc = col % RR;
-                            if (j >= J0 && j < J0 + 32) sel[j - J0] = (cc == c) ? r[n] : sel[j - J0];
+                            if (j >= J0 && j < J0 + NJ) sel[j - J0] = (cc == c) ? r[n] : sel[j - J0];
                         }
                     }
                     tc_fence_before_sync();
                     tc_mbar_arrive(&sh.acc_empty[buf]);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) gsum[j] += (double)__uint_as_float(sel[j]);
+                    for (int j = 0; j < NJ; ++j) gsum[j] += (double)__uint_as_float(sel[j]);
                 }
             };
+            // (two chunks: up to 64 gradients, 32 per warp set; three: up to 42, 21 per set; four and more: one set)
             using std::integral_constant;
+            typedef integral_constant<int, 0> I0;
             const bool upper = WIDE && warp > kMmaWarp;
-            if (!upper) {
-                switch (R) {
-                    case 2: drain_all(integral_constant<int, 2>(), integral_constant<int, 0>()); break;
-                    case 3: drain_all(integral_constant<int, 3>(), integral_constant<int, 0>()); break;
-                    case 4: drain_all(integral_constant<int, 4>(), integral_constant<int, 0>()); break;
-                    case 5: drain_all(integral_constant<int, 5>(), integral_constant<int, 0>()); break;
-                    case 6: drain_all(integral_constant<int, 6>(), integral_constant<int, 0>()); break;
-                    default: drain_all(integral_constant<int, 7>(), integral_constant<int, 0>()); break;
+            if constexpr (WIDE) {
+                if (R == 2) {
+                    if (!upper) drain_all(integral_constant<int, 2>(), I0(), integral_constant<int, 32>());
+                    else drain_all(integral_constant<int, 2>(), integral_constant<int, 32>(), integral_constant<int, 32>());
+                } else {
+                    if (!upper) drain_all(integral_constant<int, 3>(), I0(), integral_constant<int, 21>());
+                    else drain_all(integral_constant<int, 3>(), integral_constant<int, 21>(), integral_constant<int, 21>());
                 }
             } else {
-                if (R == 2) drain_all(integral_constant<int, 2>(), integral_constant<int, 32>());
-                else drain_all(integral_constant<int, 3>(), integral_constant<int, 32>());
+                switch (R) {
+                    case 4: drain_all(integral_constant<int, 4>(), I0(), integral_constant<int, 32>()); break;
+                    case 5: drain_all(integral_constant<int, 5>(), I0(), integral_constant<int, 25>()); break;
+                    case 6: drain_all(integral_constant<int, 6>(), I0(), integral_constant<int, 21>()); break;
+                    default: drain_all(integral_constant<int, 7>(), I0(), integral_constant<int, 18>()); break;
+                }
             }
         }
     }
@@ -531,11 +541,14 @@ gram_tc_kernel(const __grid_constant__ GramTcArgs a, const __grid_constant__ CUt
     double *red = reinterpret_cast<double *>(tiles);
     if (warp < 4 || warp > kMmaWarp) {
         const int row = epi_q * 32 + lane;               // row of the 128 x 128 result
-        if constexpr (TMA) {
+        if constexpr (GM) {
             const int i = row / R, c = row % R;
-            const int j0 = (WIDE && warp > kMmaWarp) ? 32 : 0;   // first gradient of this warp set's columns
+            // (the same split of the gradients between the warp sets as in the drain)
+            const int per_set = WIDE ? (R == 2 ? 32 : 21) : 32;
+            const int j0 = (WIDE && warp > kMmaWarp) ? per_set : 0;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) red[((size_t)c * Kp + i) * Kp + j0 + j] = gsum[j];
+            for (int j = 0; j < 32; ++j)
+                if (j < per_set && j0 + j < Kp) red[((size_t)c * Kp + i) * Kp + j0 + j] = gsum[j];
         } else {
             const int c = row / Kp, i = row % Kp;
             const int off = c * Kp - epi_col0;           // where this chunk's block starts in the loaded columns
